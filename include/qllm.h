@@ -1,0 +1,236 @@
+/*
+ * qllm.h -- C ABI of the B200 (sm_100a) inference hot path of a QLLM quantized
+ * linear layer (QLLM, arXiv 2310.08041).
+ *
+ * The path:  LayerNorm -> channel reassembly -> per-token asymmetric b-bit
+ * quantization  (one fused kernel, qllm_reassemble_quant), then a low-bit
+ * integer GEMM against offline-reassembled, per-output-channel quantized
+ * weights with a dequantizing epilogue (qllm_qgemm).  The reassembly map and
+ * the transformed weights are produced on the host by qllm_build_reassembly.
+ *
+ * LETTERS.  This header uses GEMM letters: M = tokens, C = K = input channels
+ * of the linear layer, N = output channels.  (The paper's Eq. 1 writes M for
+ * input channels, N for output channels and L for the sequence length.)
+ *
+ * CONVENTIONS.  Every function returns an int status: QLLM_OK (0) or a negative
+ * QLLM_ERR_* code; nothing throws.  "device" pointers are CUDA global memory of
+ * the device that is current when the call is made; "host" pointers are plain
+ * host memory.  The caller owns every buffer it passes; the library keeps no
+ * caller pointer after a call returns (device work may still be in flight on
+ * `stream`, so buffers must stay valid until that stream reaches the call).
+ * `stream` is a cudaStream_t passed as void* (NULL = default stream).  Device
+ * calls are asynchronous on `stream`, never synchronize, and launch nothing when
+ * they return an error found by argument checks.  Main device tensors (x, codes,
+ * w_codes, out) must be 16-byte aligned (QLLM_ERR_ALIGN otherwise).  There is
+ * no CPU fallback: without a usable CUDA device the device calls fail with
+ * QLLM_ERR_CUDA.
+ */
+#ifndef QLLM_H_
+#define QLLM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes -------------------------------------------------------- */
+#define QLLM_OK               0
+#define QLLM_ERR_NULL        (-1)  /* a required pointer is NULL                         */
+#define QLLM_ERR_SHAPE       (-2)  /* M < 0, C/K/N <= 0, odd channel count for 4-bit ...  */
+#define QLLM_ERR_BITS        (-3)  /* bit-width not in {4, 6, 8}                          */
+#define QLLM_ERR_DTYPE       (-4)  /* dtype selector not in {QLLM_F32, QLLM_BF16}         */
+#define QLLM_ERR_MAP         (-5)  /* reassembly map malformed (host-side checks only)   */
+#define QLLM_ERR_INFEASIBLE  (-6)  /* builder cannot bring the channel count back to C   */
+#define QLLM_ERR_CUDA        (-7)  /* CUDA runtime error; see qllm_last_cuda_error()      */
+#define QLLM_ERR_TIMEOUT     (-8)  /* a bounded device-side wait expired                  */
+#define QLLM_ERR_ALIGN       (-9)  /* a main device tensor is not 16-byte aligned         */
+#define QLLM_ERR_UNSUPPORTED (-10) /* size beyond a documented limit                      */
+#define QLLM_ERR_NOMEM       (-11) /* allocation failed                                   */
+
+#define QLLM_F32  0
+#define QLLM_BF16 1
+
+/* ==========================================================================
+ * 1. Fused pre-GEMM kernel                        (device, asynchronous)
+ * ==========================================================================
+ * For every token row m of x[M][C]:
+ *
+ *   y   = LayerNorm(x_m)            y_k = (x_k - mean) / sqrt(var + ln_eps) * gamma_k + beta_k,
+ *                                   biased variance over the C channels.  LayerNorm is the
+ *                                   non-linear layer in front of the projection that makes a
+ *                                   runtime reassembly step necessary (Sec. 4.3, "Inference
+ *                                   efficiency"); fusing it with the reassembly is the
+ *                                   paper's stated future work (Sec. 6).
+ *   x'_c = sum_{j in [map_ptr[c], map_ptr[c+1])} map_coef[j] * y[map_src[j]],   c = 0..C-1
+ *                                   channel disassembly (Eq. 3: an outlier channel becomes T
+ *                                   rows (src = i, coef = 1/T)) and channel assembly (Eq. 4:
+ *                                   a merged set becomes one row listing its members with
+ *                                   coef = 1/|set|) in one sparse map with exactly C rows.
+ *   quantize x' per token (Eq. 2):  alpha = (max x' - min x') / (2^bits - 1),
+ *                                   zero  = -round(min x' / alpha),
+ *                                   q_c   = clamp(round(x'_c / alpha) + zero, 0, 2^bits - 1),
+ *                                   round = nearest, ties to even.  A constant row takes
+ *                                   alpha = |value| (1 if the value is 0).
+ *
+ *  x         device, [M][C] row-major, float32 (x_dtype = QLLM_F32) or bfloat16 (QLLM_BF16)
+ *  ln_gamma  device float[C];  ln_beta device float[C] or NULL (= 0)
+ *  map_ptr   device int32[C+1], map_src device int32[nnz], map_coef device float[nnz];
+ *            rows non-empty, 0 <= src < C.  The map is NOT validated on the device: use
+ *            qllm_validate_map on the host copy if it does not come from the builder.
+ *  bits      4, 6 or 8
+ *  codes     device out.  bits = 4: uint8[M][C/2], byte k holds channel 2k in its low nibble
+ *            and channel 2k+1 in its high nibble (C must be even).  bits = 6 or 8: uint8[M][C].
+ *  a_scale   device out float[M]  (alpha)
+ *  a_zero    device out float[M]  (zero-point, integer-valued)
+ *  a_rowsum  device out int32[M] or NULL: sum_c q_c, needed by the GEMM epilogue
+ *  M = 0 is a successful no-op.  C <= 65536.
+ */
+int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C,
+                          const float* ln_gamma, const float* ln_beta, float ln_eps,
+                          const int32_t* map_ptr, const int32_t* map_src, const float* map_coef,
+                          int bits, uint8_t* codes, float* a_scale, float* a_zero,
+                          int32_t* a_rowsum, void* stream);
+
+/* ==========================================================================
+ * 2. Low-bit integer GEMM with dequantizing epilogue   (device, asynchronous)
+ * ==========================================================================
+ * Eq. 1 evaluated on quantized operands, Y = quant(X') quant(W') (Sec. 4.1.3),
+ * activations quantized per token and weights per output channel (Sec. 5,
+ * implementation details):
+ *
+ *   acc[m][n] = sum_k qa[m][k] * qw[n][k]                                   (int32, exact)
+ *   I[m][n]   = acc - w_zero[n]*a_rowsum[m] - a_zero[m]*w_colsum[n] + K*a_zero[m]*w_zero[n]
+ *   out[m][n] = a_scale[m] * w_scale[n] * I[m][n] + bias[n]
+ *
+ * which is Eq. 2 inverted on both operands: sum_k a_s(qa - za) * w_s(qw - zw).
+ *
+ *  codes     device, activations as written by qllm_reassemble_quant with bits = a_bits
+ *  w_codes   device, [N][K/2] packed like `codes` (w_bits = 4) or uint8[N][K] (6, 8)
+ *  w_scale, w_zero   device float[N];  w_colsum device int32[N] = sum_k qw[n][k]
+ *  bias      device float[N] or NULL
+ *  out       device, [M][N] row-major, float32 or bfloat16 (round to nearest even)
+ *  a_rowsum  device int32[M], or NULL: the row sums are then computed by a pre-pass into a
+ *            library-owned scratch buffer (grown with cudaMalloc when M exceeds what earlier
+ *            calls needed, so pass a_rowsum on allocation-free paths).
+ *  K must be even when either operand is 4-bit.  |I| must fit an int32.
+ *  Dispatch: M <= 16 takes a weight-streaming kernel (weights read once); larger M takes the
+ *  tensor-core kernel when the shape allows it, else a plain kernel.
+ */
+int qllm_qgemm(const uint8_t* codes, const float* a_scale, const float* a_zero,
+               const uint8_t* w_codes, const float* w_scale, const float* w_zero,
+               const int32_t* w_colsum, const float* bias, void* out,
+               int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype,
+               const int32_t* a_rowsum, void* stream);
+
+/* Debug twin of qllm_qgemm: writes the raw int32 accumulators acc[M][N] (same dispatch and
+ * kernels, epilogue replaced by a plain store), so that the integer sum can be compared bit
+ * for bit with a reference. */
+int qllm_qgemm_acc(const uint8_t* codes, const uint8_t* w_codes, int32_t* acc,
+                   int64_t M, int N, int K, int a_bits, int w_bits, void* stream);
+
+/* ==========================================================================
+ * 3. Calibration statistic                        (device, asynchronous)
+ * ==========================================================================
+ * absmax[k] = max(absmax[k], max_m |LayerNorm(x_m)_k|): the per-channel maximum of the layer
+ * input that Algorithm 1 starts from ("max value of each channel").  absmax must be
+ * zero-filled before the first call; calls accumulate, so calibration batches can be streamed.
+ */
+int qllm_calib_absmax(const void* x, int x_dtype, int64_t M, int C,
+                      const float* ln_gamma, const float* ln_beta, float ln_eps,
+                      float* absmax, void* stream);
+
+/* ==========================================================================
+ * 4. Offline builder                                   (host only, synchronous)
+ * ==========================================================================
+ * Turns per-channel calibration maxima into the reassembly map and the transformed,
+ * quantized weights of one linear layer:
+ *
+ *   T_i = max(1, ceil(absmax_i / theta))                     sub-channel count, Sec. 4.1.1
+ *   expanded list: channel i -> T_i consecutive entries x_i / T_i (Eq. 3); E = sum(T_i - 1)
+ *   E merges by bipartite soft matching (Appendix A): eligible entries (not born from
+ *   disassembly, Sec. 4.1.2) at even list positions form set A, at odd positions set B;
+ *   each a picks the b with the smallest |absmax_a - absmax_b| (ties: lowest position); the E
+ *   shortest edges are kept (ties: lowest a); a joins b's set, which stays at b's position and
+ *   carries the mean of its members (Eq. 4); merged a's are removed.  When one round cannot
+ *   supply E merges, all of A is merged and further rounds run on the shortened list.
+ *   W'[n][c] = sum_{j in row c} W[n][src_j]  (+ (A B)[c][n], the low-rank correction of
+ *   Sec. 4.2, folded in before quantization), then Eq. 2 per output channel n.
+ *
+ *  calib_absmax  host float[C];  theta > 0
+ *  W             host float[N][C] (output-channel major); N > 0
+ *  lr_A, lr_B    host float[C][r] (reassembled channel order) and float[r][N]; both NULL = none
+ *  w_bits        4, 6 or 8
+ *  out           receives a handle owned by the caller; release with qllm_free_reassembly
+ * Errors: QLLM_ERR_INFEASIBLE when no eligible pair is left before the count is back to C.
+ */
+typedef struct qllm_reassembly qllm_reassembly_t;
+
+int qllm_build_reassembly(const float* calib_absmax, int C, float theta,
+                          const float* W, int N,
+                          const float* lr_A, const float* lr_B, int r,
+                          int w_bits, qllm_reassembly_t** out);
+void qllm_free_reassembly(qllm_reassembly_t* h);
+
+/* Borrowed host pointers into the handle (valid until qllm_free_reassembly). */
+int qllm_reassembly_map(const qllm_reassembly_t* h, const int32_t** map_ptr,
+                        const int32_t** map_src, const float** map_coef, int64_t* nnz);
+int qllm_reassembly_weights(const qllm_reassembly_t* h, const uint8_t** w_codes, int64_t* w_bytes,
+                            const float** w_scale, const float** w_zero,
+                            const int32_t** w_colsum);
+/* stats[0] = E (channels added by disassembly = merges done), stats[1] = rows with more than
+ * one member, stats[2] = matching rounds, stats[3] = C, stats[4] = N, stats[5] = w_bits */
+int qllm_reassembly_stats(const qllm_reassembly_t* h, int64_t stats[6]);
+
+/* Host-side structural check of a map: ptr[0] = 0, rows non-empty and monotone, 0 <= src < C. */
+int qllm_validate_map(const int32_t* map_ptr, const int32_t* map_src, int C, int64_t nnz);
+
+/* theta = nearest-rank percentile of the channel maxima: sorted ascending, element
+ * ceil(pct * C) - 1.  Returns 0 on bad arguments. */
+float qllm_theta_percentile(const float* absmax, int C, double pct);
+/* A theta for which disassembly adds exactly `extra` channels: the midpoint of the interval of
+ * thresholds on which E(theta) = extra.  Returns 0 when that interval is empty. */
+float qllm_theta_for_extra(const float* absmax, int C, int extra);
+
+/* ==========================================================================
+ * 5. Layer object: device-resident map, weights and workspace
+ * ==========================================================================
+ * Convenience for callers that hold host data: uploads a built reassembly to the current
+ * device once and runs sections 1 + 2 back to back.  All allocation happens in
+ * qllm_layer_create; the forward calls allocate nothing.
+ *  x_dtype/out_dtype  QLLM_F32 or QLLM_BF16;  max_M = largest token count of a forward call
+ *  ln_gamma host float[C]; ln_beta host float[C] or NULL; bias host float[N] or NULL
+ */
+typedef struct qllm_layer qllm_layer_t;
+
+int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const float* ln_beta,
+                      float ln_eps, const float* bias, int a_bits, int x_dtype, int out_dtype,
+                      int64_t max_M, qllm_layer_t** out);
+void qllm_layer_destroy(qllm_layer_t* layer);
+/* x, out: device.  Asynchronous on stream. */
+int qllm_layer_forward(qllm_layer_t* layer, const void* x, int64_t M, void* out, void* stream);
+/* x, out: HOST (pinned memory makes the copies asynchronous).  Copies x to the device, runs the
+ * path, copies out back and waits for the stream. */
+int qllm_layer_forward_host(qllm_layer_t* layer, const void* x_host, int64_t M, void* out_host,
+                            void* stream);
+/* Borrowed DEVICE pointers of the layer's quantized-activation workspace of the last forward. */
+int qllm_layer_workspace(qllm_layer_t* layer, uint8_t** codes, float** a_scale, float** a_zero,
+                         int32_t** a_rowsum);
+
+/* ==========================================================================
+ * 6. Diagnostics
+ * ========================================================================== */
+const char* qllm_status_string(int status);
+/* Last cudaError_t seen by this library on the calling thread (0 = none). */
+int qllm_last_cuda_error(void);
+/* Reads (and clears) the device-side status word of the current device: QLLM_OK, or
+ * QLLM_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last poll.
+ * Synchronizes the device. */
+int qllm_poll_status(void);
+/* Number of kernel launches issued by this library in this process (all threads). */
+int64_t qllm_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QLLM_H_ */
