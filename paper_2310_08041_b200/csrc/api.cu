@@ -1,0 +1,291 @@
+// extern "C" entry points of the device side: argument checks, dispatch, the layer
+// object, diagnostics.  Every step of the path runs in this library's kernels.
+
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "common.h"
+
+namespace qllm {
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<int64_t> g_launch_count{0};
+
+// Device-side status word: kernels with bounded waits set it when a wait expires.
+__device__ int g_status_word = 0;
+
+int* device_status_word() {
+    int* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_status_word);
+    if (e != cudaSuccess) { cuda_fail(e); return nullptr; }
+    return p;
+}
+
+namespace {
+
+// Library-owned scratch for activation row sums when the caller passes none
+// (one buffer per device, grown on demand, never shrunk).
+struct RowsumScratch {
+    int32_t* ptr = nullptr;
+    int64_t cap = 0;
+};
+std::mutex g_scratch_mu;
+RowsumScratch g_scratch[64];
+
+int rowsum_scratch(int64_t M, int32_t** out) {
+    int dev = 0;
+    QLLM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return QLLM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    RowsumScratch& s = g_scratch[dev];
+    if (s.cap < M) {
+        if (s.ptr) QLLM_CUDA_TRY(cudaFree(s.ptr));
+        s.ptr = nullptr; s.cap = 0;
+        int64_t want = M < 4096 ? 4096 : M;
+        QLLM_CUDA_TRY(cudaMalloc(&s.ptr, size_t(want) * sizeof(int32_t)));
+        s.cap = want;
+    }
+    *out = s.ptr;
+    return QLLM_OK;
+}
+
+int check_gemm_shape(int64_t M, int N, int K, int a_bits, int w_bits) {
+    if (!bits_ok(a_bits) || !bits_ok(w_bits)) return QLLM_ERR_BITS;
+    if (M < 0 || N <= 0 || K <= 0) return QLLM_ERR_SHAPE;
+    if ((a_bits == 4 || w_bits == 4) && (K & 1)) return QLLM_ERR_SHAPE;
+    return QLLM_OK;
+}
+
+int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
+                  const EpilogueArgs& ep, cudaStream_t st) {
+    if (M == 0) return QLLM_OK;
+    if (M <= 16 && qgemm_decode_supported(M, N, K, a_bits, w_bits))
+        return launch_qgemm_decode(a, w, M, N, K, a_bits, w_bits, ep, st);
+    if (qgemm_tc_supported(M, N, K, a_bits, w_bits))
+        return launch_qgemm_tc(a, w, M, N, K, a_bits, w_bits, ep, st);
+    return launch_qgemm_plain(a, w, M, N, K, a_bits, w_bits, ep, st);
+}
+
+}  // namespace
+}  // namespace qllm
+
+using namespace qllm;
+
+struct qllm_layer {
+    int C = 0, N = 0, a_bits = 0, w_bits = 0, x_dtype = 0, out_dtype = 0;
+    int64_t max_M = 0, nnz = 0;
+    float eps = 0.f;
+    // device buffers
+    float *gamma = nullptr, *beta = nullptr, *bias = nullptr, *coef = nullptr;
+    int32_t *ptr = nullptr, *src = nullptr, *w_colsum = nullptr, *a_rowsum = nullptr;
+    uint8_t *w_codes = nullptr, *codes = nullptr;
+    float *w_scale = nullptr, *w_zero = nullptr, *a_scale = nullptr, *a_zero = nullptr;
+    void *x_dev = nullptr, *out_dev = nullptr;   // staging for the host-buffer entry point
+    std::vector<void*> owned;
+};
+
+namespace {
+template <typename T>
+int dev_alloc(qllm_layer* L, T** p, size_t count) {
+    void* q = nullptr;
+    cudaError_t e = cudaMalloc(&q, count * sizeof(T) ? count * sizeof(T) : 16);
+    if (e != cudaSuccess) { cuda_fail(e); return e == cudaErrorMemoryAllocation ? QLLM_ERR_NOMEM : QLLM_ERR_CUDA; }
+    L->owned.push_back(q);
+    *p = static_cast<T*>(q);
+    return QLLM_OK;
+}
+template <typename T>
+int dev_upload(qllm_layer* L, T** p, const T* host, size_t count) {
+    int rc = dev_alloc(L, p, count);
+    if (rc != QLLM_OK) return rc;
+    QLLM_CUDA_TRY(cudaMemcpy(*p, host, count * sizeof(T), cudaMemcpyHostToDevice));
+    return QLLM_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
+                          const float* ln_beta, float ln_eps, const int32_t* map_ptr,
+                          const int32_t* map_src, const float* map_coef, int bits, uint8_t* codes,
+                          float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream) {
+    if (!bits_ok(bits)) return QLLM_ERR_BITS;
+    if (!dtype_ok(x_dtype)) return QLLM_ERR_DTYPE;
+    if (M < 0 || C <= 0 || C > 49152 || (bits == 4 && (C & 1))) return QLLM_ERR_SHAPE;
+    if (M == 0) return QLLM_OK;
+    if (!x || !ln_gamma || !map_ptr || !map_src || !map_coef || !codes || !a_scale || !a_zero)
+        return QLLM_ERR_NULL;
+    if (!aligned16(x) || !aligned16(codes)) return QLLM_ERR_ALIGN;
+    return launch_reassemble_quant(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, map_ptr, map_src,
+                                   map_coef, bits, codes, a_scale, a_zero, a_rowsum,
+                                   static_cast<cudaStream_t>(stream));
+}
+
+int qllm_calib_absmax(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
+                      const float* ln_beta, float ln_eps, float* absmax, void* stream) {
+    if (!dtype_ok(x_dtype)) return QLLM_ERR_DTYPE;
+    if (M < 0 || C <= 0 || C > 24576) return QLLM_ERR_SHAPE;
+    if (M == 0) return QLLM_OK;
+    if (!x || !ln_gamma || !absmax) return QLLM_ERR_NULL;
+    if (!aligned16(x)) return QLLM_ERR_ALIGN;
+    return launch_calib_absmax(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, absmax,
+                               static_cast<cudaStream_t>(stream));
+}
+
+int qllm_qgemm(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
+               const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias,
+               void* out, int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype,
+               const int32_t* a_rowsum, void* stream) {
+    int rc = check_gemm_shape(M, N, K, a_bits, w_bits);
+    if (rc != QLLM_OK) return rc;
+    if (!dtype_ok(out_dtype)) return QLLM_ERR_DTYPE;
+    if (M == 0) return QLLM_OK;
+    if (!codes || !a_scale || !a_zero || !w_codes || !w_scale || !w_zero || !w_colsum || !out)
+        return QLLM_ERR_NULL;
+    if (!aligned16(codes) || !aligned16(w_codes) || !aligned16(out)) return QLLM_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!a_rowsum) {
+        int32_t* scratch = nullptr;
+        rc = rowsum_scratch(M, &scratch);
+        if (rc != QLLM_OK) return rc;
+        rc = launch_rowsum(codes, M, K, a_bits, scratch, st);
+        if (rc != QLLM_OK) return rc;
+        a_rowsum = scratch;
+    }
+    EpilogueArgs ep{a_scale, a_zero, a_rowsum, w_scale, w_zero, w_colsum, bias, out, out_dtype, 0};
+    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, st);
+}
+
+int qllm_qgemm_acc(const uint8_t* codes, const uint8_t* w_codes, int32_t* acc, int64_t M, int N, int K,
+                   int a_bits, int w_bits, void* stream) {
+    int rc = check_gemm_shape(M, N, K, a_bits, w_bits);
+    if (rc != QLLM_OK) return rc;
+    if (M == 0) return QLLM_OK;
+    if (!codes || !w_codes || !acc) return QLLM_ERR_NULL;
+    if (!aligned16(codes) || !aligned16(w_codes) || !aligned16(acc)) return QLLM_ERR_ALIGN;
+    EpilogueArgs ep{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, acc, QLLM_F32, 1};
+    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------- layer
+int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const float* ln_beta,
+                      float ln_eps, const float* bias, int a_bits, int x_dtype, int out_dtype,
+                      int64_t max_M, qllm_layer_t** out) {
+    if (!h || !ln_gamma || !out) return QLLM_ERR_NULL;
+    if (!bits_ok(a_bits)) return QLLM_ERR_BITS;
+    if (!dtype_ok(x_dtype) || !dtype_ok(out_dtype)) return QLLM_ERR_DTYPE;
+    if (max_M <= 0) return QLLM_ERR_SHAPE;
+    const int32_t *ptr, *src; const float* coef; int64_t nnz;
+    const uint8_t* wc; int64_t wbytes; const float *ws, *wz; const int32_t* wcs;
+    int64_t st[6];
+    qllm_reassembly_map(h, &ptr, &src, &coef, &nnz);
+    qllm_reassembly_weights(h, &wc, &wbytes, &ws, &wz, &wcs);
+    qllm_reassembly_stats(h, st);
+    const int C = int(st[3]), N = int(st[4]), w_bits = int(st[5]);
+    if (a_bits == 4 && (C & 1)) return QLLM_ERR_SHAPE;
+    qllm_layer* L = new (std::nothrow) qllm_layer();
+    if (!L) return QLLM_ERR_NOMEM;
+    L->C = C; L->N = N; L->a_bits = a_bits; L->w_bits = w_bits; L->x_dtype = x_dtype;
+    L->out_dtype = out_dtype; L->max_M = max_M; L->nnz = nnz; L->eps = ln_eps;
+    int rc = QLLM_OK;
+    auto step = [&](int r) { if (rc == QLLM_OK) rc = r; };
+    step(dev_upload(L, &L->gamma, ln_gamma, size_t(C)));
+    if (ln_beta) step(dev_upload(L, &L->beta, ln_beta, size_t(C)));
+    if (bias) step(dev_upload(L, &L->bias, bias, size_t(N)));
+    step(dev_upload(L, &L->ptr, ptr, size_t(C) + 1));
+    step(dev_upload(L, &L->src, src, size_t(nnz)));
+    step(dev_upload(L, &L->coef, coef, size_t(nnz)));
+    step(dev_upload(L, &L->w_codes, wc, size_t(wbytes)));
+    step(dev_upload(L, &L->w_scale, ws, size_t(N)));
+    step(dev_upload(L, &L->w_zero, wz, size_t(N)));
+    step(dev_upload(L, &L->w_colsum, wcs, size_t(N)));
+    step(dev_alloc(L, &L->codes, size_t(max_M) * size_t(code_row_bytes(C, a_bits))));
+    step(dev_alloc(L, &L->a_scale, size_t(max_M)));
+    step(dev_alloc(L, &L->a_zero, size_t(max_M)));
+    step(dev_alloc(L, &L->a_rowsum, size_t(max_M)));
+    const size_t xb = x_dtype == QLLM_F32 ? 4 : 2, ob = out_dtype == QLLM_F32 ? 4 : 2;
+    uint8_t *xd = nullptr, *od = nullptr;
+    step(dev_alloc(L, &xd, size_t(max_M) * size_t(C) * xb));
+    step(dev_alloc(L, &od, size_t(max_M) * size_t(N) * ob));
+    L->x_dev = xd; L->out_dev = od;
+    if (rc != QLLM_OK) { qllm_layer_destroy(L); return rc; }
+    *out = L;
+    return QLLM_OK;
+}
+
+void qllm_layer_destroy(qllm_layer_t* L) {
+    if (!L) return;
+    for (void* p : L->owned) cudaFree(p);
+    delete L;
+}
+
+int qllm_layer_forward(qllm_layer_t* L, const void* x, int64_t M, void* out, void* stream) {
+    if (!L || !x || !out) return QLLM_ERR_NULL;
+    if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
+    int rc = qllm_reassemble_quant(x, L->x_dtype, M, L->C, L->gamma, L->beta, L->eps, L->ptr, L->src,
+                                   L->coef, L->a_bits, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream);
+    if (rc != QLLM_OK) return rc;
+    return qllm_qgemm(L->codes, L->a_scale, L->a_zero, L->w_codes, L->w_scale, L->w_zero, L->w_colsum,
+                      L->bias, out, M, L->N, L->C, L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum, stream);
+}
+
+int qllm_layer_forward_host(qllm_layer_t* L, const void* x_host, int64_t M, void* out_host, void* stream) {
+    if (!L || !x_host || !out_host) return QLLM_ERR_NULL;
+    if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
+    if (M == 0) return QLLM_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t xb = L->x_dtype == QLLM_F32 ? 4 : 2, ob = L->out_dtype == QLLM_F32 ? 4 : 2;
+    QLLM_CUDA_TRY(cudaMemcpyAsync(L->x_dev, x_host, size_t(M) * L->C * xb, cudaMemcpyHostToDevice, st));
+    int rc = qllm_layer_forward(L, L->x_dev, M, L->out_dev, stream);
+    if (rc != QLLM_OK) return rc;
+    QLLM_CUDA_TRY(cudaMemcpyAsync(out_host, L->out_dev, size_t(M) * L->N * ob, cudaMemcpyDeviceToHost, st));
+    QLLM_CUDA_TRY(cudaStreamSynchronize(st));
+    return QLLM_OK;
+}
+
+int qllm_layer_workspace(qllm_layer_t* L, uint8_t** codes, float** a_scale, float** a_zero, int32_t** a_rowsum) {
+    if (!L) return QLLM_ERR_NULL;
+    if (codes) *codes = L->codes;
+    if (a_scale) *a_scale = L->a_scale;
+    if (a_zero) *a_zero = L->a_zero;
+    if (a_rowsum) *a_rowsum = L->a_rowsum;
+    return QLLM_OK;
+}
+
+// ---------------------------------------------------------------------------- diagnostics
+const char* qllm_status_string(int s) {
+    switch (s) {
+        case QLLM_OK: return "ok";
+        case QLLM_ERR_NULL: return "a required pointer is NULL";
+        case QLLM_ERR_SHAPE: return "invalid shape";
+        case QLLM_ERR_BITS: return "bit-width must be 4, 6 or 8";
+        case QLLM_ERR_DTYPE: return "dtype must be QLLM_F32 or QLLM_BF16";
+        case QLLM_ERR_MAP: return "malformed reassembly map";
+        case QLLM_ERR_INFEASIBLE: return "channel count cannot be restored by assembly";
+        case QLLM_ERR_CUDA: return "CUDA error (see qllm_last_cuda_error)";
+        case QLLM_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case QLLM_ERR_ALIGN: return "device tensor not 16-byte aligned";
+        case QLLM_ERR_UNSUPPORTED: return "size beyond a documented limit";
+        case QLLM_ERR_NOMEM: return "out of memory";
+        default: return "unknown status";
+    }
+}
+
+int qllm_last_cuda_error(void) { return g_last_cuda_error; }
+
+int qllm_poll_status(void) {
+    int v = 0;
+    QLLM_CUDA_TRY(cudaDeviceSynchronize());
+    QLLM_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_status_word, sizeof(int)));
+    if (v != 0) {
+        const int zero = 0;
+        QLLM_CUDA_TRY(cudaMemcpyToSymbol(g_status_word, &zero, sizeof(int)));
+        return QLLM_ERR_TIMEOUT;
+    }
+    return QLLM_OK;
+}
+
+int64_t qllm_launch_count(void) { return g_launch_count.load(); }
+
+}  // extern "C"

@@ -1,0 +1,79 @@
+// Shared host-side plumbing of the library: error bookkeeping, launch counter,
+// argument-check helpers.  No kernel code lives here.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "../../include/qllm.h"
+
+namespace qllm {
+
+extern thread_local int g_last_cuda_error;
+extern std::atomic<int64_t> g_launch_count;
+
+inline int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = static_cast<int>(e);
+    return QLLM_ERR_CUDA;
+}
+
+// Records a launch and turns a launch-time error into a status.
+inline int after_launch(int n_launches = 1) {
+    g_launch_count.fetch_add(n_launches, std::memory_order_relaxed);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    return QLLM_OK;
+}
+
+#define QLLM_CUDA_TRY(expr)                                   \
+    do {                                                      \
+        cudaError_t _e = (expr);                              \
+        if (_e != cudaSuccess) return ::qllm::cuda_fail(_e);  \
+    } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool bits_ok(int b) { return b == 4 || b == 6 || b == 8; }
+inline bool dtype_ok(int d) { return d == QLLM_F32 || d == QLLM_BF16; }
+// Bytes of one row of K codes at the given bit-width (4-bit codes are packed two per byte).
+inline int64_t code_row_bytes(int K, int bits) { return bits == 4 ? K / 2 : K; }
+
+// Device-side status word (one per loaded library image and device).
+int* device_status_word();          // device address, or nullptr on failure (error recorded)
+
+// ---- kernels' host launchers (each returns a status) ----------------------
+struct EpilogueArgs {
+    const float* a_scale;
+    const float* a_zero;
+    const int32_t* a_rowsum;
+    const float* w_scale;
+    const float* w_zero;
+    const int32_t* w_colsum;
+    const float* bias;      // may be null
+    void* out;              // [M][N] f32 / bf16, or int32 when raw_acc
+    int out_dtype;          // QLLM_F32 / QLLM_BF16
+    int raw_acc;            // 1: store int32 accumulators, ignore everything else
+};
+
+int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
+                            const float* beta, float eps, const int32_t* ptr, const int32_t* src,
+                            const float* coef, int bits, uint8_t* codes, float* a_scale,
+                            float* a_zero, int32_t* a_rowsum, cudaStream_t st);
+int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
+                                    const float* beta, float eps, const int32_t* ptr, const int32_t* src,
+                                    const float* coef, int bits, uint8_t* codes, float* a_scale,
+                                    float* a_zero, int32_t* a_rowsum, cudaStream_t st);
+int launch_calib_absmax(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
+                        const float* beta, float eps, float* absmax, cudaStream_t st);
+int launch_rowsum(const uint8_t* codes, int64_t M, int K, int bits, int32_t* rowsum, cudaStream_t st);
+int launch_qgemm_plain(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
+                       int w_bits, const EpilogueArgs& ep, cudaStream_t st);
+int launch_qgemm_decode(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
+                        int w_bits, const EpilogueArgs& ep, cudaStream_t st);
+bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits);
+int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
+                    int w_bits, const EpilogueArgs& ep, cudaStream_t st);
+bool qgemm_decode_supported(int64_t M, int N, int K, int a_bits, int w_bits);
+
+}  // namespace qllm

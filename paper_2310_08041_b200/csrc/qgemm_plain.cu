@@ -1,0 +1,105 @@
+// Shape-agnostic integer GEMM with the dequantizing epilogue, and the row code-sum
+// pre-pass.  One thread per output element, operands read code by code: this is the
+// path for shapes the tensor-core and weight-streaming kernels do not take (odd K,
+// unaligned rows) and the on-device cross-check of those kernels.
+
+#include "common.h"
+#include "epilogue.cuh"
+
+namespace qllm {
+
+namespace {
+
+__device__ __forceinline__ int code_at(const uint8_t* row, int k, int bits) {
+    if (bits == 4) {
+        const int b = row[k >> 1];
+        return (k & 1) ? (b >> 4) : (b & 0xF);
+    }
+    return row[k];
+}
+
+// Eight consecutive codes starting at k (k % 8 == 0) as two words of four byte lanes:
+// lanes of `even` = codes k, k+2, k+4, k+6; lanes of `odd` = codes k+1, k+3, k+5, k+7.
+// Both operands use the same order, so the dot product is unchanged.
+__device__ __forceinline__ void eight_codes(const uint8_t* row, int k, int bits, uint32_t& even, uint32_t& odd) {
+    if (bits == 4) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(row + (k >> 1));
+        even = w & 0x0F0F0F0Fu;
+        odd = (w >> 4) & 0x0F0F0F0Fu;
+    } else {
+        const uint2 w = *reinterpret_cast<const uint2*>(row + k);
+        even = __byte_perm(w.x, w.y, 0x6420);
+        odd = __byte_perm(w.x, w.y, 0x7531);
+    }
+}
+
+template <bool WORDS>
+__global__ void __launch_bounds__(256)
+qgemm_plain_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ w, int64_t M, int N, int K,
+                   int a_bits, int w_bits, EpilogueArgs ep) {
+    const int n = blockIdx.x * 32 + (threadIdx.x & 31);
+    const int64_t m = int64_t(blockIdx.y) * 8 + (threadIdx.x >> 5);
+    if (n >= N || m >= M) return;
+    const uint8_t* arow = a + m * (a_bits == 4 ? K / 2 : K);
+    const uint8_t* wrow = w + int64_t(n) * (w_bits == 4 ? K / 2 : K);
+    int acc = 0;
+    if (WORDS) {
+        for (int k = 0; k < K; k += 8) {
+            uint32_t ae, ao, we, wo;
+            eight_codes(arow, k, a_bits, ae, ao);
+            eight_codes(wrow, k, w_bits, we, wo);
+            acc = int(__dp4a(ae, we, uint32_t(acc)));      // unsigned lanes
+            acc = int(__dp4a(ao, wo, uint32_t(acc)));
+        }
+    } else {
+        for (int k = 0; k < K; ++k) acc += code_at(arow, k, a_bits) * code_at(wrow, k, w_bits);
+    }
+    if (ep.raw_acc) {
+        static_cast<int32_t*>(ep.out)[m * N + n] = acc;
+        return;
+    }
+    const RowTerm r = make_row_term(ep.a_scale, ep.a_zero, ep.a_rowsum, m);
+    const ColTerm c = make_col_term(ep.w_scale, ep.w_zero, ep.w_colsum, ep.bias, K, n);
+    const float o = dequant(acc, r, c);
+    if (ep.out_dtype == QLLM_F32) static_cast<float*>(ep.out)[m * N + n] = o;
+    else static_cast<__nv_bfloat16*>(ep.out)[m * N + n] = __float2bfloat16_rn(o);
+}
+
+// One warp per row: sum of the row's codes.
+__global__ void __launch_bounds__(256)
+rowsum_kernel(const uint8_t* __restrict__ codes, int64_t M, int K, int bits, int32_t* __restrict__ rowsum) {
+    const int64_t m = int64_t(blockIdx.x) * 8 + (threadIdx.x >> 5);
+    if (m >= M) return;
+    const int lane = threadIdx.x & 31;
+    const int nbytes = bits == 4 ? K / 2 : K;
+    const uint8_t* row = codes + m * nbytes;
+    int s = 0;
+    for (int i = lane; i < nbytes; i += 32) {
+        const int b = row[i];
+        s += bits == 4 ? (b & 0xF) + (b >> 4) : b;
+    }
+    s = __reduce_add_sync(0xffffffffu, s);
+    if (lane == 0) rowsum[m] = s;
+}
+
+}  // namespace
+
+int launch_rowsum(const uint8_t* codes, int64_t M, int K, int bits, int32_t* rowsum, cudaStream_t st) {
+    if (M == 0) return QLLM_OK;
+    rowsum_kernel<<<unsigned((M + 7) / 8), 256, 0, st>>>(codes, M, K, bits, rowsum);
+    return after_launch();
+}
+
+int launch_qgemm_plain(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
+                       const EpilogueArgs& ep, cudaStream_t st) {
+    if (M == 0) return QLLM_OK;
+    if ((M + 7) / 8 > 65535) return QLLM_ERR_UNSUPPORTED;
+    dim3 grid(unsigned((N + 31) / 32), unsigned((M + 7) / 8));
+    // word loads need 4-byte aligned rows for both operands
+    const bool words = (K % 8 == 0);
+    if (words) qgemm_plain_kernel<true><<<grid, 256, 0, st>>>(a, w, M, N, K, a_bits, w_bits, ep);
+    else qgemm_plain_kernel<false><<<grid, 256, 0, st>>>(a, w, M, N, K, a_bits, w_bits, ep);
+    return after_launch();
+}
+
+}  // namespace qllm
