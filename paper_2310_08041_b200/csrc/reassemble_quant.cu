@@ -1,14 +1,360 @@
-// Dispatch of the fused pre-GEMM stage.
+// Fused pre-GEMM kernel: LayerNorm -> channel reassembly -> per-token asymmetric
+// quantization (QLLM Eq. 2-4; the fusion the paper leaves as future work, Sec. 6).
+//
+// HBM-bound: every token row of x is read once and its codes written once.  Design:
+//  * persistent CTAs, C / CPT threads each; a thread owns CPT output channels for every
+//    token its CTA processes, so the reassembly map is read ONCE per CTA into registers:
+//    per channel the first two entries (source offset, coefficient * gamma) and the bias
+//    term sum_j coef_j * beta[src_j].  Per token the only shared-memory traffic is the
+//    centred row d = x - mean (written once, 4 B / channel) and the gathers from it.
+//        x'_c = rstd * sum_j (coef_j gamma[src_j]) d[src_j] + sum_j coef_j beta[src_j]
+//    Rows with more than two entries (a channel that absorbed several others) add their
+//    tail from the CSR arrays in a short per-thread loop.
+//  * 128-bit coalesced loads of the row, next row prefetched into registers.
+//  * ownership is by channel pairs (2p, 2p+1), p = t + NT*i, so a thread packs whole bytes
+//    of 4-bit codes; lanes 16-31 keep their pairs swapped in registers so that the two
+//    gathers of a pair hit different banks across the two half-warps.
+//  * three CTA reductions per token (sum, sum of squares, min/max) through shared memory,
+//    parity-double-buffered so each costs one barrier.
+//  * rounding by the 1.5 * 2^23 magic constant (nearest-even, as cvt.rni), saturating
+//    cvt.pack for the clamp and the nibble / byte packing.
+// Shapes outside the specialisation (C not a multiple of 32*CPT, C > 8192) take the
+// shape-agnostic kernel.
+
+#include <cuda_bf16.h>
+
 #include "common.h"
+#include "device_utils.cuh"
 
 namespace qllm {
+
+namespace {
+
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
+constexpr int kMagicBits = 0x4B400000;
+
+template <typename XT> struct RowLoad;
+template <> struct RowLoad<__nv_bfloat16> { static constexpr int PER_CHUNK = 8; };
+template <> struct RowLoad<float> { static constexpr int PER_CHUNK = 4; };
+
+__device__ __forceinline__ float redux_min(float v) {
+    float r;
+    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ float redux_max(float v) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+// d = sat_u4(a) << 4 | sat_u4(b) | c << 8
+__device__ __forceinline__ uint32_t pack_sat_u4(int a, int b, uint32_t c) {
+    uint32_t d;
+    asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// d = sat_u8(a) << 8 | sat_u8(b) | c << 16
+__device__ __forceinline__ uint32_t pack_sat_u8(int a, int b, uint32_t c) {
+    uint32_t d;
+    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+// Sum over the CTA of one value per warp already stored in red[0..nw4) (zero padded to a
+// multiple of four).  Same order in every thread, so all threads hold identical bits.
+__device__ __forceinline__ float sum_of(const float* red, int nw4) {
+    float s = 0.f;
+    for (int w = 0; w < nw4; w += 4) {
+        const float4 q = *reinterpret_cast<const float4*>(red + w);
+        s += (q.x + q.y) + (q.z + q.w);
+    }
+    return s;
+}
+
+template <int CPT, typename XT>
+__global__ void __launch_bounds__(512)
+reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* __restrict__ gamma,
+                      const float* __restrict__ beta, float eps, const int32_t* __restrict__ ptr,
+                      const int32_t* __restrict__ src, const float* __restrict__ coef, int bits,
+                      uint8_t* __restrict__ codes, float* __restrict__ a_scale, float* __restrict__ a_zero,
+                      int32_t* __restrict__ a_rowsum) {
+    constexpr int PER = RowLoad<XT>::PER_CHUNK;
+    constexpr int NCH = CPT / PER;               // 16-byte chunks of the row per thread
+    constexpr int NP = CPT / 2;                  // channel pairs per thread
+    extern __shared__ __align__(16) uint8_t smem_bytes[];
+    float* d = reinterpret_cast<float*>(smem_bytes);           // [C] centred row
+    float* red = d + C;                                        // [2][4][32] per-warp partials
+    int* redi = reinterpret_cast<int*>(red + 2 * 4 * 32);      // [2][32] code-sum partials
+
+    const int t = threadIdx.x, NT = blockDim.x, lane = t & 31, warp = t >> 5;
+    const int nw = NT >> 5, nw4 = (nw + 3) & ~3;
+    const bool rot = lane >= 16;
+    const float invC = 1.0f / float(C);
+    const float qmax = float((1 << bits) - 1);
+
+    for (int i = t; i < 2 * 4 * 32 + 2 * 32; i += NT) red[i] = 0.f;   // also zeroes redi (bit pattern 0)
+
+    // ---- map -> registers (once per CTA) ------------------------------------------------
+    uint32_t off[CPT];        // byte offsets into d: entry 0 in the low half, entry 1 in the high half
+    float cg0[CPT], cg1[CPT], bias[CPT];
+    uint64_t longlist = 0;    // slots (4 bits each) whose row has more than two entries
+    int nlong = 0;
+    {
+        // three rounds of independent loads (row bounds, entries, gamma/beta) instead of
+        // CPT dependent chains: the set-up is latency-bound and runs once per CTA
+        int j0[CPT], len[CPT];
+#pragma unroll
+        for (int slot = 0; slot < CPT; ++slot) {
+            const int c = 2 * (t + NT * (slot >> 1)) + ((slot & 1) ^ int(rot));
+            j0[slot] = __ldg(ptr + c);
+            len[slot] = __ldg(ptr + c + 1) - j0[slot];
+        }
+        int s0[CPT], s1[CPT];
+        float c0[CPT], c1[CPT];
+#pragma unroll
+        for (int slot = 0; slot < CPT; ++slot) {
+            const int j1 = j0[slot] + (len[slot] >= 2 ? 1 : 0);
+            s0[slot] = __ldg(src + j0[slot]);
+            s1[slot] = __ldg(src + j1);
+            c0[slot] = __ldg(coef + j0[slot]);
+            c1[slot] = __ldg(coef + j1);
+        }
+#pragma unroll
+        for (int slot = 0; slot < CPT; ++slot) {
+            if (len[slot] < 2) c1[slot] = 0.f;
+            cg0[slot] = c0[slot] * __ldg(gamma + s0[slot]);
+            cg1[slot] = c1[slot] * __ldg(gamma + s1[slot]);
+            float b = 0.f;
+            if (beta) b = fmaf(c1[slot], __ldg(beta + s1[slot]), c0[slot] * __ldg(beta + s0[slot]));
+            bias[slot] = b;
+            off[slot] = uint32_t(s0[slot] * 4) | (uint32_t(s1[slot] * 4) << 16);
+        }
+#pragma unroll
+        for (int slot = 0; slot < CPT; ++slot) {
+            if (len[slot] > 2) {
+                longlist |= uint64_t(slot) << (4 * nlong);
+                ++nlong;
+                if (beta)
+                    for (int j = j0[slot] + 2; j < j0[slot] + len[slot]; ++j)
+                        bias[slot] = fmaf(coef[j], beta[src[j]], bias[slot]);
+            }
+        }
+    }
+
+    // ---- token loop ---------------------------------------------------------------------
+    uint4 raw[NCH];
+    int64_t m = blockIdx.x;
+    if (m < M) {
+#pragma unroll
+        for (int j = 0; j < NCH; ++j)
+            raw[j] = *reinterpret_cast<const uint4*>(x + m * C + PER * (t + NT * j));
+    }
+    __syncthreads();
+    int par = 0;
+    int64_t m_prev = -1;
+    for (; m < M; m += gridDim.x, par ^= 1) {
+        float* rsum = red + par * 128;
+        float* rsq = rsum + 32;
+        float* rlo = rsum + 64;
+        float* rhi = rsum + 96;
+        // -- row to fp32, mean
+        float xv[CPT];
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            if constexpr (PER == 8) {
+                const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    xv[8 * j + 2 * k] = __uint_as_float(w[k] << 16);
+                    xv[8 * j + 2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u);
+                }
+            } else {
+                xv[4 * j] = __uint_as_float(raw[j].x); xv[4 * j + 1] = __uint_as_float(raw[j].y);
+                xv[4 * j + 2] = __uint_as_float(raw[j].z); xv[4 * j + 3] = __uint_as_float(raw[j].w);
+            }
+        }
+        const int64_t m_next = m + gridDim.x;
+        if (m_next < M) {
+#pragma unroll
+            for (int j = 0; j < NCH; ++j)
+                raw[j] = *reinterpret_cast<const uint4*>(x + m_next * C + PER * (t + NT * j));
+        }
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < CPT; ++i) s += xv[i];
+        s = warp_sum(s);
+        if (lane == 0) rsum[warp] = s;
+        __syncthreads();                                               // S1
+        const float mean = sum_of(rsum, nw4) * invC;
+        if (t == 0 && m_prev >= 0 && a_rowsum) {                       // code sum of the previous token
+            const int* ri = redi + (par ^ 1) * 32;
+            int tot = 0;
+            for (int w = 0; w < nw; ++w) tot += ri[w];
+            a_rowsum[m_prev] = tot;
+        }
+        // -- centred row to shared memory, variance
+        float sq = 0.f;
+#pragma unroll
+        for (int i = 0; i < CPT; ++i) {
+            xv[i] -= mean;
+            sq = fmaf(xv[i], xv[i], sq);
+        }
+#pragma unroll
+        for (int j = 0; j < NCH; ++j) {
+            float* dst = d + PER * (t + NT * j);
+#pragma unroll
+            for (int k = 0; k < PER; k += 4)
+                *reinterpret_cast<float4*>(dst + k) =
+                    make_float4(xv[PER * j + k], xv[PER * j + k + 1], xv[PER * j + k + 2], xv[PER * j + k + 3]);
+        }
+        sq = warp_sum(sq);
+        if (lane == 0) rsq[warp] = sq;
+        __syncthreads();                                               // S2: d visible
+        const float var = sum_of(rsq, nw4) * invC;
+        const float rstd = 1.0f / sqrtf(var + eps);
+        // -- reassembly: gather from d with the register-resident map
+        const char* dbytes = reinterpret_cast<const char*>(d);
+        float v[CPT];
+#pragma unroll
+        for (int slot = 0; slot < CPT; ++slot) {
+            const float a0 = *reinterpret_cast<const float*>(dbytes + (off[slot] & 0xFFFFu));
+            const float a1 = *reinterpret_cast<const float*>(dbytes + (off[slot] >> 16));
+            const float acc = fmaf(cg1[slot], a1, cg0[slot] * a0);
+            v[slot] = acc;
+        }
+        for (int k = 0; k < nlong; ++k) {                              // rows with > 2 entries (rare)
+            const int slot = int((longlist >> (4 * k)) & 15u);
+            const int c = 2 * (t + NT * (slot >> 1)) + ((slot & 1) ^ int(rot));
+            float e = 0.f;
+            for (int j = ptr[c] + 2; j < ptr[c + 1]; ++j) {
+                const int sj = src[j];
+                e = fmaf(coef[j] * gamma[sj], d[sj], e);
+            }
+#pragma unroll
+            for (int q = 0; q < CPT; ++q)
+                if (q == slot) v[q] += e;
+        }
+        float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+        for (int slot = 0; slot < CPT; ++slot) {
+            v[slot] = fmaf(rstd, v[slot], bias[slot]);
+            lo = fminf(lo, v[slot]);
+            hi = fmaxf(hi, v[slot]);
+        }
+        lo = redux_min(lo);
+        hi = redux_max(hi);
+        if (lane == 0) { rlo[warp] = lo; rhi[warp] = hi; }
+        __syncthreads();                                               // S3
+        for (int w = 0; w < nw; ++w) { lo = fminf(lo, rlo[w]); hi = fmaxf(hi, rhi[w]); }
+        // -- Eq. 2
+        float alpha = (hi - lo) / qmax;
+        if (!(hi > lo)) alpha = lo != 0.f ? fabsf(lo) : 1.f;
+        const float inv = 1.0f / alpha;
+        const float zero = -rintf(lo / alpha);
+        const bool big = fmaxf(fabsf(lo), fabsf(hi)) * inv >= 2097152.f || fabsf(zero) >= 2097152.f;
+        const int zadd = int(zero) - kMagicBits;
+        int n[CPT];
+        if (!big) {
+#pragma unroll
+            for (int slot = 0; slot < CPT; ++slot)
+                n[slot] = __float_as_int(fmaf(v[slot], inv, kMagic)) + zadd;
+        } else {
+#pragma unroll
+            for (int slot = 0; slot < CPT; ++slot) {
+                const float q = fminf(fmaxf(rintf(v[slot] * inv) + zero, 0.f), qmax);
+                n[slot] = int(q);
+            }
+        }
+        int csum = 0;
+        if (bits == 4) {
+            // one byte per pair: low nibble = even channel.  Pack as held, then swap the nibbles
+            // on the lanes that keep their pairs swapped.
+            uint32_t w[NP / 4];
+#pragma unroll
+            for (int g = 0; g < NP / 4; ++g) {
+                uint32_t p = 0;
+#pragma unroll
+                for (int i = 3; i >= 0; --i) p = pack_sat_u4(n[2 * (4 * g + i) + 1], n[2 * (4 * g + i)], p);
+                const uint32_t sw = ((p << 4) & 0xF0F0F0F0u) | ((p >> 4) & 0x0F0F0F0Fu);
+                w[g] = rot ? sw : p;
+                const uint32_t nib = (p & 0x0F0F0F0Fu) + ((p >> 4) & 0x0F0F0F0Fu);
+                csum = int(__dp4a(nib, 0x01010101u, uint32_t(csum)));
+            }
+            uint8_t* out = codes + m * (C / 2) + t;
+#pragma unroll
+            for (int i = 0; i < NP; ++i) out[NT * i] = uint8_t(w[i >> 2] >> (8 * (i & 3)));
+        } else {
+            const int top = int(qmax);
+            uint16_t* out = reinterpret_cast<uint16_t*>(codes + m * C) + t;
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const int e = rot ? n[2 * i + 1] : n[2 * i];
+                const int o = rot ? n[2 * i] : n[2 * i + 1];
+                const uint32_t p = pack_sat_u8(min(o, top), min(e, top), 0);
+                out[NT * i] = uint16_t(p);
+                csum += int(p & 0xFFu) + int(p >> 8);
+            }
+        }
+        if (t == 0) { a_scale[m] = alpha; a_zero[m] = zero; }
+        csum = __reduce_add_sync(0xffffffffu, csum);
+        if (lane == 0) redi[par * 32 + warp] = csum;
+        m_prev = m;
+    }
+    __syncthreads();
+    if (t == 0 && m_prev >= 0 && a_rowsum) {
+        const int* ri = redi + (par ^ 1) * 32;
+        int tot = 0;
+        for (int w = 0; w < nw; ++w) tot += ri[w];
+        a_rowsum[m_prev] = tot;
+    }
+}
+
+int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            n = 148;
+    }
+    return n;
+}
+
+template <int CPT, typename XT>
+int launch_fast(const void* x, int64_t M, int C, const float* gamma, const float* beta, float eps,
+                const int32_t* ptr, const int32_t* src, const float* coef, int bits, uint8_t* codes,
+                float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
+    auto kern = reassemble_quant_fast<CPT, XT>;
+    const int nt = C / CPT;
+    const size_t smem = size_t(C) * 4 + (2 * 4 * 32 + 2 * 32) * 4;
+    if (smem > 48 * 1024)
+        QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
+    int per_sm = 0;
+    QLLM_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, nt, smem));
+    if (per_sm < 1) per_sm = 1;
+    const int grid = int(std::min<int64_t>(M, int64_t(sm_count()) * per_sm));
+    kern<<<grid, nt, smem, st>>>(static_cast<const XT*>(x), M, C, gamma, beta, eps, ptr, src, coef, bits,
+                                 codes, a_scale, a_zero, a_rowsum);
+    return after_launch();
+}
+
+}  // namespace
 
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                             const float* coef, int bits, uint8_t* codes, float* a_scale,
                             float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
-    return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits,
-                                           codes, a_scale, a_zero, a_rowsum, st);
+    const bool bf = x_dtype == QLLM_BF16;
+    if (C % 512 == 0 && C <= 8192) {
+        return bf ? launch_fast<16, __nv_bfloat16>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st)
+                  : launch_fast<16, float>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st);
+    }
+    if (C % 256 == 0 && C <= 4096) {
+        return bf ? launch_fast<8, __nv_bfloat16>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st)
+                  : launch_fast<8, float>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st);
+    }
+    return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
+                                           a_scale, a_zero, a_rowsum, st);
 }
 
 }  // namespace qllm
