@@ -30,6 +30,7 @@ namespace qllm {
 
 namespace {
 
+constexpr int kVirt = 256;                     // rows with > 2 entries served through virtual slots
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr int kMagicBits = 0x4B400000;
 
@@ -71,8 +72,8 @@ __device__ __forceinline__ float sum_of(const float* red, int nw4) {
     return s;
 }
 
-template <int CPT, typename XT>
-__global__ void __launch_bounds__(512)
+template <int CPT, int NTT, typename XT>
+__global__ void __launch_bounds__(NTT ? NTT : 512, (NTT && NTT <= 256) ? 2 : 1)
 reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* __restrict__ gamma,
                       const float* __restrict__ beta, float eps, const int32_t* __restrict__ ptr,
                       const int32_t* __restrict__ src, const float* __restrict__ coef, int bits,
@@ -82,17 +83,21 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
     constexpr int NCH = CPT / PER;               // 16-byte chunks of the row per thread
     constexpr int NP = CPT / 2;                  // channel pairs per thread
     extern __shared__ __align__(16) uint8_t smem_bytes[];
-    float* d = reinterpret_cast<float*>(smem_bytes);           // [C] centred row
-    float* red = d + C;                                        // [2][4][32] per-warp partials
+    float* red = reinterpret_cast<float*>(smem_bytes);         // [2][4][32] per-warp partials
     int* redi = reinterpret_cast<int*>(red + 2 * 4 * 32);      // [2][32] code-sum partials
+    int* vrow = redi + 2 * 32;                                 // [kVirt] rows served by virtual slots
+    int* vcount = vrow + kVirt;                                // [4] counter (+ padding)
+    float* d = reinterpret_cast<float*>(vcount + 4);           // [C + kVirt] centred row + virtual slots
 
-    const int t = threadIdx.x, NT = blockDim.x, lane = t & 31, warp = t >> 5;
+    const int t = threadIdx.x, NT = NTT ? NTT : int(blockDim.x), lane = t & 31, warp = t >> 5;
     const int nw = NT >> 5, nw4 = (nw + 3) & ~3;
     const bool rot = lane >= 16;
     const float invC = 1.0f / float(C);
     const float qmax = float((1 << bits) - 1);
+    const float inv_qmax = 1.0f / qmax;
 
-    for (int i = t; i < 2 * 4 * 32 + 2 * 32; i += NT) red[i] = 0.f;   // also zeroes redi (bit pattern 0)
+    for (int i = t; i < 2 * 4 * 32 + 2 * 32 + kVirt + 4; i += NT) red[i] = 0.f;   // zero bit pattern for the int arrays too
+    __syncthreads();
 
     // ---- map -> registers (once per CTA) ------------------------------------------------
     uint32_t off[CPT];        // byte offsets into d: entry 0 in the low half, entry 1 in the high half
@@ -132,11 +137,20 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
 #pragma unroll
         for (int slot = 0; slot < CPT; ++slot) {
             if (len[slot] > 2) {
-                longlist |= uint64_t(slot) << (4 * nlong);
-                ++nlong;
                 if (beta)
                     for (int j = j0[slot] + 2; j < j0[slot] + len[slot]; ++j)
                         bias[slot] = fmaf(coef[j], beta[src[j]], bias[slot]);
+                // Entries 1.. of this row are summed once per token into virtual slot d[C + vi] by
+                // one thread; the owner then reads that slot as its second entry with weight 1.
+                const int vi = atomicAdd(vcount, 1);
+                if (vi < kVirt) {
+                    vrow[vi] = 2 * (t + NT * (slot >> 1)) + ((slot & 1) ^ int(rot));
+                    cg1[slot] = 1.0f;
+                    off[slot] = (off[slot] & 0xFFFFu) | (uint32_t((C + vi) * 4) << 16);
+                } else {                       // more long rows than virtual slots: per-thread tail loop
+                    longlist |= uint64_t(slot) << (4 * nlong);
+                    ++nlong;
+                }
             }
         }
     }
@@ -150,6 +164,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             raw[j] = *reinterpret_cast<const uint4*>(x + m * C + PER * (t + NT * j));
     }
     __syncthreads();
+    const int nvirt = min(*vcount, kVirt);
     int par = 0;
     int64_t m_prev = -1;
     for (; m < M; m += gridDim.x, par ^= 1) {
@@ -211,7 +226,20 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
         if (lane == 0) rsq[warp] = sq;
         __syncthreads();                                               // S2: d visible
         const float var = sum_of(rsq, nw4) * invC;
-        const float rstd = 1.0f / sqrtf(var + eps);
+        const float rstd = rsqrtf(var + eps);        // a common factor of the whole row: its last-bit
+                                                     // error rescales alpha with the row, codes unchanged
+        if (nvirt > 0) {                             // uniform over the CTA
+            for (int vi = t; vi < nvirt; vi += NT) {
+                const int c = vrow[vi];
+                float e = 0.f;
+                for (int j = __ldg(ptr + c) + 1; j < __ldg(ptr + c + 1); ++j) {
+                    const int sj = __ldg(src + j);
+                    e = fmaf(__ldg(coef + j) * __ldg(gamma + sj), d[sj], e);
+                }
+                d[C + vi] = e;
+            }
+            __syncthreads();                                           // S2b
+        }
         // -- reassembly: gather from d with the register-resident map
         const char* dbytes = reinterpret_cast<const char*>(d);
         float v[CPT];
@@ -245,12 +273,23 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
         hi = redux_max(hi);
         if (lane == 0) { rlo[warp] = lo; rhi[warp] = hi; }
         __syncthreads();                                               // S3
-        for (int w = 0; w < nw; ++w) { lo = fminf(lo, rlo[w]); hi = fmaxf(hi, rhi[w]); }
+        for (int w = 0; w < nw4; w += 4) {          // padding holds 0: restored below from real warps
+            const float4 a = *reinterpret_cast<const float4*>(rlo + w);
+            const float4 b = *reinterpret_cast<const float4*>(rhi + w);
+            if (w + 3 < nw) {
+                lo = fminf(fminf(lo, fminf(a.x, a.y)), fminf(a.z, a.w));
+                hi = fmaxf(fmaxf(hi, fmaxf(b.x, b.y)), fmaxf(b.z, b.w));
+            } else {
+                lo = fminf(lo, a.x); hi = fmaxf(hi, b.x);
+                if (w + 1 < nw) { lo = fminf(lo, a.y); hi = fmaxf(hi, b.y); }
+                if (w + 2 < nw) { lo = fminf(lo, a.z); hi = fmaxf(hi, b.z); }
+            }
+        }
         // -- Eq. 2
-        float alpha = (hi - lo) / qmax;
+        float alpha = (hi - lo) * inv_qmax;
         if (!(hi > lo)) alpha = lo != 0.f ? fabsf(lo) : 1.f;
-        const float inv = 1.0f / alpha;
-        const float zero = -rintf(lo / alpha);
+        const float inv = __frcp_rn(alpha);
+        const float zero = -rintf(lo * inv);
         const bool big = fmaxf(fabsf(lo), fabsf(hi)) * inv >= 2097152.f || fabsf(zero) >= 2097152.f;
         const int zadd = int(zero) - kMagicBits;
         int n[CPT];
@@ -320,13 +359,13 @@ int sm_count() {
     return n;
 }
 
-template <int CPT, typename XT>
+template <int CPT, int NTT, typename XT>
 int launch_fast(const void* x, int64_t M, int C, const float* gamma, const float* beta, float eps,
                 const int32_t* ptr, const int32_t* src, const float* coef, int bits, uint8_t* codes,
                 float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
-    auto kern = reassemble_quant_fast<CPT, XT>;
+    auto kern = reassemble_quant_fast<CPT, NTT, XT>;
     const int nt = C / CPT;
-    const size_t smem = size_t(C) * 4 + (2 * 4 * 32 + 2 * 32) * 4;
+    const size_t smem = size_t(C + kVirt) * 4 + (2 * 4 * 32 + 2 * 32 + kVirt + 4) * 4;
     if (smem > 48 * 1024)
         QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     int per_sm = 0;
@@ -340,19 +379,21 @@ int launch_fast(const void* x, int64_t M, int C, const float* gamma, const float
 
 }  // namespace
 
+#define QLLM_RQ_ARGS x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st
+
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                             const float* coef, int bits, uint8_t* codes, float* a_scale,
                             float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
     const bool bf = x_dtype == QLLM_BF16;
-    if (C % 512 == 0 && C <= 8192) {
-        return bf ? launch_fast<16, __nv_bfloat16>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st)
-                  : launch_fast<16, float>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st);
-    }
-    if (C % 256 == 0 && C <= 4096) {
-        return bf ? launch_fast<8, __nv_bfloat16>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st)
-                  : launch_fast<8, float>(x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st);
-    }
+    // LLaMA hidden sizes get compile-time thread counts (immediate offsets, unrolled reductions)
+    if (bf && C == 4096) return launch_fast<16, 256, __nv_bfloat16>(QLLM_RQ_ARGS);
+    if (bf && C == 5120) return launch_fast<16, 320, __nv_bfloat16>(QLLM_RQ_ARGS);
+    if (bf && C == 8192) return launch_fast<16, 512, __nv_bfloat16>(QLLM_RQ_ARGS);
+    if (C % 512 == 0 && C <= 8192)
+        return bf ? launch_fast<16, 0, __nv_bfloat16>(QLLM_RQ_ARGS) : launch_fast<16, 0, float>(QLLM_RQ_ARGS);
+    if (C % 256 == 0 && C <= 4096)
+        return bf ? launch_fast<8, 0, __nv_bfloat16>(QLLM_RQ_ARGS) : launch_fast<8, 0, float>(QLLM_RQ_ARGS);
     return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
                                            a_scale, a_zero, a_rowsum, st);
 }
