@@ -84,7 +84,7 @@ extern "C" {
  *  a_scale   device out float[M]  (alpha)
  *  a_zero    device out float[M]  (zero-point, integer-valued)
  *  a_rowsum  device out int32[M] or NULL: sum_c q_c, needed by the GEMM epilogue
- *  M = 0 is a successful no-op.  C <= 65536.
+ *  M = 0 is a successful no-op.  C <= 49152 (the normalised row is held in shared memory).
  */
 int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C,
                           const float* ln_gamma, const float* ln_beta, float ln_eps,
@@ -135,6 +135,7 @@ int qllm_qgemm_acc(const uint8_t* codes, const uint8_t* w_codes, int32_t* acc,
  * absmax[k] = max(absmax[k], max_m |LayerNorm(x_m)_k|): the per-channel maximum of the layer
  * input that Algorithm 1 starts from ("max value of each channel").  absmax must be
  * zero-filled before the first call; calls accumulate, so calibration batches can be streamed.
+ * C <= 24576.
  */
 int qllm_calib_absmax(const void* x, int x_dtype, int64_t M, int C,
                       const float* ln_gamma, const float* ln_beta, float ln_eps,

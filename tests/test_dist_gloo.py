@@ -1,0 +1,61 @@
+"""N > 1 host logic on CPU: two gloo ranks shard a token batch, agree on coverage, and combine
+their timings with a max-reduction (what `bench.py --gpus N` does over NCCL)."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2310_08041_b200.shard import max_over_ranks, token_shard
+
+
+def test_token_shard_partitions_rows():
+    for M in (0, 1, 7, 64, 2048, 4097):
+        for world in (1, 2, 3, 8):
+            cover = []
+            for r in range(world):
+                s, n = token_shard(M, r, world)
+                cover.extend(range(s, s + n))
+            assert cover == list(range(M))
+            sizes = [token_shard(M, r, world)[1] for r in range(world)]
+            assert max(sizes) - min(sizes) <= 1
+
+
+def _worker(rank, world, port, M, out_q):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    start, count = token_shard(M, rank, world)
+    # each rank "processes" its rows: here, marks them
+    mine = torch.zeros(M, dtype=torch.int32)
+    mine[start:start + count] = rank + 1
+    dist.all_reduce(mine, op=dist.ReduceOp.SUM)
+    t = max_over_ranks(10.0 + rank)           # rank-dependent step time
+    total = torch.tensor([count], dtype=torch.int64)
+    dist.all_reduce(total)
+    out_q.put((rank, mine.numpy().copy(), t, int(total.item())))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_shard_and_reduce():
+    world, M = 2, 101
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, M, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = [q.get(timeout=120) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, marks, t, total in res:
+        assert t == 11.0                      # max over ranks, identical on every rank
+        assert total == M
+        s0, n0 = token_shard(M, 0, world)
+        assert np.all(marks[:n0] == 1) and np.all(marks[n0:] == 2)   # every row owned exactly once
