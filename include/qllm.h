@@ -123,6 +123,28 @@ int qllm_qgemm(const uint8_t* codes, const float* a_scale, const float* a_zero,
                int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype,
                const int32_t* a_rowsum, void* stream);
 
+/* Allocation-free variant of qllm_qgemm (the paper has no counterpart; it exists for callers
+ * that cannot call cudaMalloc: code inside a caller-managed memory pool or a latency-critical
+ * serving loop, where an allocation may synchronise the device or fail, and processes that
+ * have given all device memory to another allocator).  It always computes the activation row
+ * sums itself, into a fixed array of QLLM_NOALLOC_MAX_M int32 (256 KiB) that is part of the
+ * library image: every GPU that loads the library holds it until the process exits.  It calls
+ * no cudaMalloc / cudaFree and no allocating library routine.
+ *  - M > QLLM_NOALLOC_MAX_M returns QLLM_ERR_UNSUPPORTED; all other arguments and errors are
+ *    those of qllm_qgemm (without a_rowsum).
+ *  - The first call on a device looks up the array's device address; make that first call
+ *    before any stream capture begins.
+ *  - All calls on a device share the one array.  Each call overwrites the M entries it uses
+ *    before reading them, so nothing from an earlier call leaks in; but two calls whose work
+ *    overlaps on the GPU (different streams) race on it: serialise them.
+ */
+#define QLLM_NOALLOC_MAX_M 65536
+int qllm_qgemm_noalloc(const uint8_t* codes, const float* a_scale, const float* a_zero,
+                       const uint8_t* w_codes, const float* w_scale, const float* w_zero,
+                       const int32_t* w_colsum, const float* bias, void* out,
+                       int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype,
+                       void* stream);
+
 /* Debug twin of qllm_qgemm: writes the raw int32 accumulators acc[M][N] (same dispatch and
  * kernels, epilogue replaced by a plain store), so that the integer sum can be compared bit
  * for bit with a reference. */

@@ -24,7 +24,7 @@ QLLM_F32, QLLM_BF16 = 0, 1
 
 # every symbol include/qllm.h declares
 EXPORTS = [
-    "qllm_reassemble_quant", "qllm_qgemm", "qllm_qgemm_acc", "qllm_calib_absmax",
+    "qllm_reassemble_quant", "qllm_qgemm", "qllm_qgemm_noalloc", "qllm_qgemm_acc", "qllm_calib_absmax",
     "qllm_build_reassembly", "qllm_free_reassembly", "qllm_reassembly_map",
     "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map",
     "qllm_theta_percentile", "qllm_theta_for_extra",
@@ -42,6 +42,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 _vp, _i, _i64, _f, _d = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_double
 _lib.qllm_reassemble_quant.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.qllm_qgemm.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.qllm_qgemm_noalloc.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i, _i, _i, _i, _i, _vp]
 _lib.qllm_qgemm_acc.argtypes = [_vp, _vp, _vp, _i64, _i, _i, _i, _i, _vp]
 _lib.qllm_calib_absmax.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp]
 _lib.qllm_build_reassembly.argtypes = [_vp, _i, _f, _vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(_vp)]
@@ -121,6 +122,19 @@ def qllm_qgemm(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, bias,
     _check(_lib.qllm_qgemm(_dp(codes), _dp(a_scale), _dp(a_zero), _dp(w_codes), _dp(w_scale), _dp(w_zero),
                            _dp(w_colsum), _dp(bias), _dp(out), M, N, K, a_bits, w_bits, _xdtype(out),
                            _dp(a_rowsum), _stream(stream)))
+
+
+QLLM_NOALLOC_MAX_M = 65536
+
+
+def qllm_qgemm_noalloc(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, bias, out, M, N, K, a_bits, w_bits,
+                       stream=None):
+    """qllm_qgemm for callers that must not allocate: the activation row sums are computed into
+    a fixed array inside the library (at most QLLM_NOALLOC_MAX_M rows), never into cudaMalloc'd
+    scratch.  Calls on one device share that array, so do not overlap them on the GPU."""
+    _check(_lib.qllm_qgemm_noalloc(_dp(codes), _dp(a_scale), _dp(a_zero), _dp(w_codes), _dp(w_scale), _dp(w_zero),
+                                   _dp(w_colsum), _dp(bias), _dp(out), M, N, K, a_bits, w_bits, _xdtype(out),
+                                   _stream(stream)))
 
 
 def qllm_qgemm_acc(codes, w_codes, acc, M, N, K, a_bits, w_bits, stream=None):
