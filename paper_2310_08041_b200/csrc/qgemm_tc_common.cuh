@@ -1,0 +1,181 @@
+// Pieces shared by the tcgen05 GEMM kernels: bounded mbarrier waits, the nibble -> byte tile
+// expansion, the dequantizing store of an accumulator chunk, tensor-map construction.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.h"
+#include "epilogue.cuh"
+#include "ptx_sm100.cuh"
+
+namespace qllm {
+namespace tc {
+
+constexpr int BM = 128;              // tile rows (tokens) per CTA = MMA M
+constexpr int BK = 128;              // codes of K per pipeline stage = one 128-byte swizzle row
+constexpr int kUnpackWarps = 8;
+constexpr int kFirstEpiWarp = 2, kFirstUnpackWarp = 6;
+constexpr long long kWaitCycles = 1ll << 32;   // ~2 s at 2 GHz
+
+struct Abort {
+    volatile int* flag;     // shared: some role gave up
+    int* status;            // global status word of the library
+};
+
+__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, const Abort& ab) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t i = 1;; ++i) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 0) {
+            if (*ab.flag) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *ab.flag = 1;
+                atomicExch(ab.status, QLLM_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+// Expand a ROWS x 64-byte tile of packed nibbles into a ROWS x 128-byte swizzled byte tile.
+// 16-byte chunk j of row r (codes 32j .. 32j+31) fills units 2j and 2j+1 of the row, each unit
+// stored at position unit ^ (r & 7).  PAIRED (both operands 4-bit): even nibbles to unit 2j,
+// odd nibbles to unit 2j+1 -- a permutation of K shared by both operands.  Otherwise (the other
+// operand holds byte codes in natural order) the nibbles are interleaved back into K order.
+template <int ROWS, bool PAIRED>
+__device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ raw, uint8_t* __restrict__ op, int t) {
+    constexpr int PER_THREAD = ROWS * 4 / (32 * kUnpackWarps);
+    static_assert(PER_THREAD * 32 * kUnpackWarps == ROWS * 4, "tile rows must split evenly over the unpack threads");
+#pragma unroll
+    for (int i = 0; i < PER_THREAD; ++i) {
+        const int q = t + i * 32 * kUnpackWarps;
+        const int r = q >> 2, j = q & 3;
+        const uint4 w = *reinterpret_cast<const uint4*>(raw + q * 16);
+        uint4 lo, hi;
+        lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
+        lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
+        lo.z = w.z & 0x0F0F0F0Fu; hi.z = (w.z >> 4) & 0x0F0F0F0Fu;
+        lo.w = w.w & 0x0F0F0F0Fu; hi.w = (w.w >> 4) & 0x0F0F0F0Fu;
+        uint4 u0 = lo, u1 = hi;
+        if (!PAIRED) {
+            u0.x = __byte_perm(lo.x, hi.x, 0x5140); u0.y = __byte_perm(lo.x, hi.x, 0x7362);
+            u0.z = __byte_perm(lo.y, hi.y, 0x5140); u0.w = __byte_perm(lo.y, hi.y, 0x7362);
+            u1.x = __byte_perm(lo.z, hi.z, 0x5140); u1.y = __byte_perm(lo.z, hi.z, 0x7362);
+            u1.z = __byte_perm(lo.w, hi.w, 0x5140); u1.w = __byte_perm(lo.w, hi.w, 0x7362);
+        }
+        uint8_t* row = op + r * 128;
+        const int sw = r & 7;
+        *reinterpret_cast<uint4*>(row + (((2 * j) ^ sw) << 4)) = u0;
+        *reinterpret_cast<uint4*>(row + (((2 * j + 1) ^ sw) << 4)) = u1;
+    }
+}
+
+
+// Epilogue of one 32-column chunk of one accumulator row: r[c] = acc[m][nb + c].  Either stores the raw
+// int32 accumulators or dequantizes with the row term and the staged column terms and stores f32 / bf16.
+// N is a multiple of 8, so 16-byte groups never straddle the end of a row.
+__device__ __forceinline__ void store_chunk(const EpilogueArgs& ep, const uint32_t (&r)[32], const int4* colterm,
+                                            const RowTerm& rt, int64_t m, int N, int nb) {
+    if (ep.raw_acc) {
+        int32_t* o = static_cast<int32_t*>(ep.out) + m * N + nb;
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+            if (nb + 4 * v < N)
+                *reinterpret_cast<int4*>(o + 4 * v) = make_int4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+        return;
+    }
+    float f[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+        const int4 ct = colterm[c];
+        const int I = int(r[c]) - ct.y * rt.rowsum - rt.zero * ct.z;
+        f[c] = fmaf(rt.scale * __int_as_float(ct.x), float(I), __int_as_float(ct.w));
+    }
+    if (ep.out_dtype == QLLM_F32) {
+        float* o = static_cast<float*>(ep.out) + m * N + nb;
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+            if (nb + 4 * v < N)
+                *reinterpret_cast<float4*>(o + 4 * v) = make_float4(f[4 * v], f[4 * v + 1], f[4 * v + 2], f[4 * v + 3]);
+    } else {
+        __nv_bfloat16* o = static_cast<__nv_bfloat16*>(ep.out) + m * N + nb;
+#pragma unroll
+        for (int v = 0; v < 4; ++v)
+            if (nb + 8 * v < N) {
+                uint4 pk;
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(f[8 * v], f[8 * v + 1]);
+                __nv_bfloat162 h1 = __floats2bfloat162_rn(f[8 * v + 2], f[8 * v + 3]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[8 * v + 4], f[8 * v + 5]);
+                __nv_bfloat162 h3 = __floats2bfloat162_rn(f[8 * v + 6], f[8 * v + 7]);
+                pk.x = *reinterpret_cast<uint32_t*>(&h0); pk.y = *reinterpret_cast<uint32_t*>(&h1);
+                pk.z = *reinterpret_cast<uint32_t*>(&h2); pk.w = *reinterpret_cast<uint32_t*>(&h3);
+                *reinterpret_cast<uint4*>(o + 8 * v) = pk;
+            }
+    }
+}
+
+// Column terms of the tile's output channels -> shared memory (scale, zero, colsum - K*zero, bias).
+__device__ __forceinline__ void stage_col_terms(const EpilogueArgs& ep, int4* colterm, int bn, int n0, int N, int K,
+                                                int et, int nthreads) {
+    if (ep.raw_acc) return;
+    for (int c = et; c < bn; c += nthreads) {
+        const int n = n0 + c;
+        int4 v = make_int4(0, 0, 0, 0);
+        if (n < N) {
+            const ColTerm ct = make_col_term(ep.w_scale, ep.w_zero, ep.w_colsum, ep.bias, K, n);
+            v = make_int4(__float_as_int(ct.scale), ct.zero, ct.corr, __float_as_int(ct.bias));
+        }
+        colterm[c] = v;
+    }
+}
+
+// ---- host side ----------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// uint8 matrix [rows][row_bytes]; box = box_rows x box_bytes; out-of-range parts read as zero.
+inline bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows,
+              uint32_t box_bytes, bool swizzle128) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {box_bytes, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+inline int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            n = 148;
+    }
+    return n;
+}
+
+
+}  // namespace tc
+}  // namespace qllm
