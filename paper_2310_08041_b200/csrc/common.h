@@ -74,6 +74,8 @@ int launch_qgemm_decode(const uint8_t* a, const uint8_t* w, int64_t M, int N, in
 bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits);
 int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
                     int w_bits, const EpilogueArgs& ep, cudaStream_t st);
+int launch_qgemm_tc_w4a4(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const EpilogueArgs& ep,
+                         cudaStream_t st);
 bool qgemm_decode_supported(int64_t M, int N, int K, int a_bits, int w_bits);
 
 }  // namespace qllm
