@@ -57,17 +57,81 @@ int check_gemm_shape(int64_t M, int N, int K, int a_bits, int w_bits) {
     return QLLM_OK;
 }
 
+// Library-owned scratch for the byte-expanded operands of large 4-bit GEMMs: one buffer per
+// (device, stream), grown on demand, never shrunk.
+struct ExpandScratch { cudaStream_t st; uint8_t* ptr; size_t cap; };
+std::vector<ExpandScratch> g_expand[64];
+
+int expand_scratch(cudaStream_t st, size_t bytes, uint8_t** out) {
+    int dev = 0;
+    QLLM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return QLLM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    ExpandScratch* e = nullptr;
+    for (auto& x : g_expand[dev]) if (x.st == st) e = &x;
+    if (!e) { g_expand[dev].push_back({st, nullptr, 0}); e = &g_expand[dev].back(); }
+    if (e->cap < bytes) {
+        if (e->ptr) QLLM_CUDA_TRY(cudaFree(e->ptr));
+        e->ptr = nullptr; e->cap = 0;
+        QLLM_CUDA_TRY(cudaMalloc(&e->ptr, bytes));
+        e->cap = bytes;
+    }
+    *out = e->ptr;
+    return QLLM_OK;
+}
+
+// Token count from which expanding 4-bit operands to bytes once per call (a bandwidth-bound pre-pass
+// over N*K + M*K codes) and running the byte-lane tensor-core kernel beats unpacking every tile in
+// shared memory, which caps the tensor pipe near 40 %.
+constexpr int64_t kExpandMinM = 512;
+
 int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
-                  const EpilogueArgs& ep, cudaStream_t st) {
+                  const EpilogueArgs& ep, cudaStream_t st, bool may_allocate) {
     if (M == 0) return QLLM_OK;
     if (M <= 16 && qgemm_decode_supported(M, N, K, a_bits, w_bits))
         return launch_qgemm_decode(a, w, M, N, K, a_bits, w_bits, ep, st);
-    if (qgemm_tc_supported(M, N, K, a_bits, w_bits))
+    if (qgemm_tc_supported(M, N, K, a_bits, w_bits)) {
+        const bool ap = a_bits == 4, wp = w_bits == 4;
+        if (may_allocate && (ap || wp) && M >= kExpandMinM) {
+            const size_t a_bytes = ap ? size_t(M) * K : 0, w_bytes = wp ? size_t(N) * K : 0;
+            uint8_t* buf = nullptr;
+            int rc = expand_scratch(st, a_bytes + w_bytes, &buf);
+            if (rc != QLLM_OK) return rc;
+            if (ap) { rc = launch_expand_codes(a, M, K, buf, st); if (rc != QLLM_OK) return rc; a = buf; }
+            if (wp) { rc = launch_expand_codes(w, N, K, buf + a_bytes, st); if (rc != QLLM_OK) return rc; w = buf + a_bytes; }
+            return launch_qgemm_tc(a, w, M, N, K, 8, 8, ep, st);
+        }
         return launch_qgemm_tc(a, w, M, N, K, a_bits, w_bits, ep, st);
+    }
     return launch_qgemm_plain(a, w, M, N, K, a_bits, w_bits, ep, st);
 }
 
 }  // namespace
+
+int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
+               const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
+               int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
+               cudaStream_t st, bool may_allocate) {
+    int rc = check_gemm_shape(M, N, K, a_bits, w_bits);
+    if (rc != QLLM_OK) return rc;
+    if (!dtype_ok(out_dtype)) return QLLM_ERR_DTYPE;
+    if (M == 0) return QLLM_OK;
+    if (!codes || !a_scale || !a_zero || !w_codes || !w_scale || !w_zero || !w_colsum || !out)
+        return QLLM_ERR_NULL;
+    if (!aligned16(codes) || !aligned16(w_codes) || !aligned16(out)) return QLLM_ERR_ALIGN;
+    if (!a_rowsum) {
+        if (!may_allocate) return QLLM_ERR_NULL;
+        int32_t* scratch = nullptr;
+        rc = rowsum_scratch(M, &scratch);
+        if (rc != QLLM_OK) return rc;
+        rc = launch_rowsum(codes, M, K, a_bits, scratch, st);
+        if (rc != QLLM_OK) return rc;
+        a_rowsum = scratch;
+    }
+    EpilogueArgs ep{a_scale, a_zero, a_rowsum, w_scale, w_zero, w_colsum, bias, out, out_dtype, 0};
+    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, st, may_allocate);
+}
+
 }  // namespace qllm
 
 using namespace qllm;
@@ -137,24 +201,8 @@ int qllm_qgemm(const uint8_t* codes, const float* a_scale, const float* a_zero, 
                const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias,
                void* out, int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype,
                const int32_t* a_rowsum, void* stream) {
-    int rc = check_gemm_shape(M, N, K, a_bits, w_bits);
-    if (rc != QLLM_OK) return rc;
-    if (!dtype_ok(out_dtype)) return QLLM_ERR_DTYPE;
-    if (M == 0) return QLLM_OK;
-    if (!codes || !a_scale || !a_zero || !w_codes || !w_scale || !w_zero || !w_colsum || !out)
-        return QLLM_ERR_NULL;
-    if (!aligned16(codes) || !aligned16(w_codes) || !aligned16(out)) return QLLM_ERR_ALIGN;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (!a_rowsum) {
-        int32_t* scratch = nullptr;
-        rc = rowsum_scratch(M, &scratch);
-        if (rc != QLLM_OK) return rc;
-        rc = launch_rowsum(codes, M, K, a_bits, scratch, st);
-        if (rc != QLLM_OK) return rc;
-        a_rowsum = scratch;
-    }
-    EpilogueArgs ep{a_scale, a_zero, a_rowsum, w_scale, w_zero, w_colsum, bias, out, out_dtype, 0};
-    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, st);
+    return gemm_entry(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, bias, out, M, N, K, a_bits,
+                      w_bits, out_dtype, a_rowsum, static_cast<cudaStream_t>(stream), true);
 }
 
 int qllm_qgemm_acc(const uint8_t* codes, const uint8_t* w_codes, int32_t* acc, int64_t M, int N, int K,
@@ -165,7 +213,7 @@ int qllm_qgemm_acc(const uint8_t* codes, const uint8_t* w_codes, int32_t* acc, i
     if (!codes || !w_codes || !acc) return QLLM_ERR_NULL;
     if (!aligned16(codes) || !aligned16(w_codes) || !aligned16(acc)) return QLLM_ERR_ALIGN;
     EpilogueArgs ep{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, acc, QLLM_F32, 1};
-    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, static_cast<cudaStream_t>(stream));
+    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, static_cast<cudaStream_t>(stream), true);
 }
 
 // ---------------------------------------------------------------------------- layer

@@ -66,6 +66,12 @@ int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C
                                     float* a_zero, int32_t* a_rowsum, cudaStream_t st);
 int launch_calib_absmax(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                         const float* beta, float eps, float* absmax, cudaStream_t st);
+int launch_expand_codes(const uint8_t* packed, int64_t rows, int K, uint8_t* bytes, cudaStream_t st);
+// The GEMM behind qllm_qgemm.  may_allocate = false keeps it on paths that never grow library scratch.
+int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
+               const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
+               int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
+               cudaStream_t st, bool may_allocate);
 int launch_rowsum(const uint8_t* codes, int64_t M, int K, int bits, int32_t* rowsum, cudaStream_t st);
 int launch_qgemm_plain(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
                        int w_bits, const EpilogueArgs& ep, cudaStream_t st);
@@ -74,8 +80,6 @@ int launch_qgemm_decode(const uint8_t* a, const uint8_t* w, int64_t M, int N, in
 bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits);
 int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
                     int w_bits, const EpilogueArgs& ep, cudaStream_t st);
-int launch_qgemm_tc_w4a4(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const EpilogueArgs& ep,
-                         cudaStream_t st);
 bool qgemm_decode_supported(int64_t M, int N, int K, int a_bits, int w_bits);
 
 }  // namespace qllm

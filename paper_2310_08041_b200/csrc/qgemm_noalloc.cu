@@ -58,7 +58,7 @@ extern "C" int qllm_qgemm_noalloc(const uint8_t* codes, const float* a_scale, co
     // every one of the M entries is overwritten, so nothing left by an earlier call is read
     rc = launch_rowsum(codes, M, K, a_bits, rowsum, static_cast<cudaStream_t>(stream));
     if (rc != QLLM_OK) return rc;
-    // with the row sums supplied, qllm_qgemm takes no allocating path
-    return qllm_qgemm(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, bias, out, M, N, K, a_bits,
-                      w_bits, out_dtype, rowsum, stream);
+    // the same GEMM as qllm_qgemm, held to the paths that never grow library scratch
+    return gemm_entry(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, bias, out, M, N, K, a_bits,
+                      w_bits, out_dtype, rowsum, static_cast<cudaStream_t>(stream), false);
 }

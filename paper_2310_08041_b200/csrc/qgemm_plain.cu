@@ -82,7 +82,35 @@ rowsum_kernel(const uint8_t* __restrict__ codes, int64_t M, int K, int bits, int
     if (lane == 0) rowsum[m] = s;
 }
 
+// Packed nibbles [rows][K/2] -> byte codes [rows][K] in natural K order.  One 16-byte chunk
+// (32 codes) per thread in, 32 contiguous bytes out; purely bandwidth-bound.
+__global__ void __launch_bounds__(256)
+expand_codes_kernel(const uint4* __restrict__ packed, int64_t chunks, uint4* __restrict__ bytes) {
+    for (int64_t i = int64_t(blockIdx.x) * 256 + threadIdx.x; i < chunks; i += int64_t(gridDim.x) * 256) {
+        const uint4 w = packed[i];
+        const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t lo = in[k] & 0x0F0F0F0Fu, hi = (in[k] >> 4) & 0x0F0F0F0Fu;
+            o[2 * k] = __byte_perm(lo, hi, 0x5140);
+            o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);
+        }
+        bytes[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+        bytes[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
 }  // namespace
+
+int launch_expand_codes(const uint8_t* packed, int64_t rows, int K, uint8_t* bytes, cudaStream_t st) {
+    const int64_t chunks = rows * (K / 32);
+    if (chunks == 0) return QLLM_OK;
+    const int grid = int(std::min<int64_t>((chunks + 255) / 256, 148 * 16));
+    expand_codes_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const uint4*>(packed), chunks,
+                                              reinterpret_cast<uint4*>(bytes));
+    return after_launch();
+}
 
 int launch_rowsum(const uint8_t* codes, int64_t M, int K, int bits, int32_t* rowsum, cudaStream_t st) {
     if (M == 0) return QLLM_OK;

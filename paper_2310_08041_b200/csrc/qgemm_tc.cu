@@ -15,8 +15,6 @@
 // the MMAs of tile i+1.  Every mbarrier wait is bounded: on expiry the kernel raises the
 // library's device status word, all roles leave their loops, TMEM is freed, and the kernel ends.
 
-#include <cstdlib>
-
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -244,11 +242,7 @@ bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits) {
 int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
                     const EpilogueArgs& ep, cudaStream_t st) {
     const bool ap = a_bits == 4, wp = w_bits == 4;
-    if (ap && wp) {
-        // QLLM_W4A4_STAGED=1 in the environment selects the TMA-staged variant (for A/B timing)
-        static const bool staged = [] { const char* e = getenv("QLLM_W4A4_STAGED"); return e && e[0] == '1'; }();
-        return staged ? launch<256, true, true>(a, w, M, N, K, ep, st) : launch_qgemm_tc_w4a4(a, w, M, N, K, ep, st);
-    }
+    if (ap && wp) return launch<256, true, true>(a, w, M, N, K, ep, st);
     if (!ap && !wp) return launch<256, false, false>(a, w, M, N, K, ep, st);
     if (ap) return launch<256, true, false>(a, w, M, N, K, ep, st);
     return launch<256, false, true>(a, w, M, N, K, ep, st);

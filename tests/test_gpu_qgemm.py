@@ -17,6 +17,7 @@ SHAPES = [
     (257, 528, 640, 6, 6), (150, 256, 5120, 6, 6), (9, 31, 77, 6, 6), (40, 64, 256, 8, 8),
     (140, 272, 512, 8, 4), (33, 80, 256, 4, 8), (200, 16, 128, 4, 4), (128, 256, 128, 4, 4),
     (8, 136, 512, 6, 6), (12, 520, 1024, 8, 4), (5, 61, 256, 4, 8), (16, 22016, 4096, 4, 4), (1, 8, 128, 4, 4),
+    (600, 272, 256, 4, 4), (520, 136, 512, 8, 4), (513, 80, 160, 4, 8),
 ]
 
 
