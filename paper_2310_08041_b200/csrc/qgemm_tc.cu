@@ -243,7 +243,19 @@ int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K,
                     const EpilogueArgs& ep, cudaStream_t st) {
     const bool ap = a_bits == 4, wp = w_bits == 4;
     if (ap && wp) return launch<256, true, true>(a, w, M, N, K, ep, st);
-    if (!ap && !wp) return launch<256, false, false>(a, w, M, N, K, ep, st);
+    if (!ap && !wp) {
+        // tile width that wastes the least of the last wave: cost ~ rounds x tile width
+        const int64_t tm = (M + BM - 1) / BM;
+        const int sms = sm_count();
+        auto cost = [&](int bn) {
+            const int64_t tiles = tm * ((N + bn - 1) / bn);
+            return ((tiles + sms - 1) / sms) * int64_t(bn + 16);   // + per-tile fill/drain overhead
+        };
+        const int64_t c256 = cost(256), c192 = cost(192), c128 = cost(128);
+        if (c256 <= c192 && c256 <= c128) return launch<256, false, false>(a, w, M, N, K, ep, st);
+        if (c192 <= c128) return launch<192, false, false>(a, w, M, N, K, ep, st);
+        return launch<128, false, false>(a, w, M, N, K, ep, st);
+    }
     if (ap) return launch<256, true, false>(a, w, M, N, K, ep, st);
     return launch<256, false, true>(a, w, M, N, K, ep, st);
 }
