@@ -232,6 +232,12 @@ int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const f
 void qllm_layer_destroy(qllm_layer_t* layer);
 /* x, out: device.  Asynchronous on stream. */
 int qllm_layer_forward(qllm_layer_t* layer, const void* x, int64_t M, void* out, void* stream);
+/* The two halves of qllm_layer_forward, for callers that time or schedule them separately:
+ * qllm_layer_reassemble_quant runs the fused pre-GEMM kernel on x[M][C] (device) into the layer's
+ * workspace; qllm_layer_qgemm multiplies that workspace (M rows of the last pre-GEMM call) with the
+ * layer's weights into out[M][N] (device).  Asynchronous on stream. */
+int qllm_layer_reassemble_quant(qllm_layer_t* layer, const void* x, int64_t M, void* stream);
+int qllm_layer_qgemm(qllm_layer_t* layer, int64_t M, void* out, void* stream);
 /* x, out: HOST (pinned memory makes the copies asynchronous).  Copies x to the device, runs the
  * path, copies out back and waits for the stream. */
 int qllm_layer_forward_host(qllm_layer_t* layer, const void* x_host, int64_t M, void* out_host,

@@ -29,6 +29,7 @@ EXPORTS = [
     "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map",
     "qllm_theta_percentile", "qllm_theta_for_extra",
     "qllm_layer_create", "qllm_layer_destroy", "qllm_layer_forward", "qllm_layer_forward_host",
+    "qllm_layer_reassemble_quant", "qllm_layer_qgemm",
     "qllm_layer_workspace",
     "qllm_status_string", "qllm_last_cuda_error", "qllm_poll_status", "qllm_launch_count",
 ]
@@ -62,6 +63,8 @@ _lib.qllm_layer_destroy.argtypes = [_vp]
 _lib.qllm_layer_destroy.restype = None
 _lib.qllm_layer_forward.argtypes = [_vp, _vp, _i64, _vp, _vp]
 _lib.qllm_layer_forward_host.argtypes = [_vp, _vp, _i64, _vp, _vp]
+_lib.qllm_layer_reassemble_quant.argtypes = [_vp, _vp, _i64, _vp]
+_lib.qllm_layer_qgemm.argtypes = [_vp, _i64, _vp, _vp]
 _lib.qllm_layer_workspace.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]
 _lib.qllm_status_string.argtypes = [_i]
 _lib.qllm_status_string.restype = ctypes.c_char_p
@@ -269,6 +272,12 @@ class Layer:
 
     def forward(self, x, out, stream=None):
         _check(_lib.qllm_layer_forward(self._h, _dp(x), x.shape[0], _dp(out), _stream(stream)))
+
+    def reassemble_quant(self, x, stream=None):
+        _check(_lib.qllm_layer_reassemble_quant(self._h, _dp(x), x.shape[0], _stream(stream)))
+
+    def qgemm(self, M, out, stream=None):
+        _check(_lib.qllm_layer_qgemm(self._h, M, _dp(out), _stream(stream)))
 
     def forward_host(self, x_host, out_host, M, stream=None):
         """x_host/out_host: host pointers (ints) or numpy arrays / pinned CPU torch tensors."""

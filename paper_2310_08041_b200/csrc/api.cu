@@ -23,6 +23,30 @@ int* device_status_word() {
 }
 
 namespace {
+std::mutex g_scratch_mu;
+struct StreamScratch { cudaStream_t st; uint8_t* ptr; size_t cap; };
+std::vector<StreamScratch> g_stream_scratch[kScratchKinds][64];
+}  // namespace
+
+int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out) {
+    int dev = 0;
+    QLLM_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || kind < 0 || kind >= kScratchKinds) return QLLM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    StreamScratch* e = nullptr;
+    for (auto& x : g_stream_scratch[kind][dev]) if (x.st == st) e = &x;
+    if (!e) { g_stream_scratch[kind][dev].push_back({st, nullptr, 0}); e = &g_stream_scratch[kind][dev].back(); }
+    if (e->cap < bytes) {
+        if (e->ptr) QLLM_CUDA_TRY(cudaFree(e->ptr));
+        e->ptr = nullptr; e->cap = 0;
+        QLLM_CUDA_TRY(cudaMalloc(&e->ptr, bytes));
+        e->cap = bytes;
+    }
+    *out = e->ptr;
+    return QLLM_OK;
+}
+
+namespace {
 
 // Library-owned scratch for activation row sums when the caller passes none
 // (one buffer per device, grown on demand, never shrunk).
@@ -30,7 +54,6 @@ struct RowsumScratch {
     int32_t* ptr = nullptr;
     int64_t cap = 0;
 };
-std::mutex g_scratch_mu;
 RowsumScratch g_scratch[64];
 
 int rowsum_scratch(int64_t M, int32_t** out) {
@@ -57,29 +80,6 @@ int check_gemm_shape(int64_t M, int N, int K, int a_bits, int w_bits) {
     return QLLM_OK;
 }
 
-// Library-owned scratch for the byte-expanded operands of large 4-bit GEMMs: one buffer per
-// (device, stream), grown on demand, never shrunk.
-struct ExpandScratch { cudaStream_t st; uint8_t* ptr; size_t cap; };
-std::vector<ExpandScratch> g_expand[64];
-
-int expand_scratch(cudaStream_t st, size_t bytes, uint8_t** out) {
-    int dev = 0;
-    QLLM_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return QLLM_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lk(g_scratch_mu);
-    ExpandScratch* e = nullptr;
-    for (auto& x : g_expand[dev]) if (x.st == st) e = &x;
-    if (!e) { g_expand[dev].push_back({st, nullptr, 0}); e = &g_expand[dev].back(); }
-    if (e->cap < bytes) {
-        if (e->ptr) QLLM_CUDA_TRY(cudaFree(e->ptr));
-        e->ptr = nullptr; e->cap = 0;
-        QLLM_CUDA_TRY(cudaMalloc(&e->ptr, bytes));
-        e->cap = bytes;
-    }
-    *out = e->ptr;
-    return QLLM_OK;
-}
-
 // Token count from which expanding 4-bit operands to bytes once per call (a bandwidth-bound pre-pass
 // over N*K + M*K codes) and running the byte-lane tensor-core kernel beats unpacking every tile in
 // shared memory, which caps the tensor pipe near 40 %.
@@ -95,7 +95,7 @@ int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, i
         if (may_allocate && (ap || wp) && M >= kExpandMinM) {
             const size_t a_bytes = ap ? size_t(M) * K : 0, w_bytes = wp ? size_t(N) * K : 0;
             uint8_t* buf = nullptr;
-            int rc = expand_scratch(st, a_bytes + w_bytes, &buf);
+            int rc = stream_scratch(kScratchExpand, st, a_bytes + w_bytes, &buf);
             if (rc != QLLM_OK) return rc;
             if (ap) { rc = launch_expand_codes(a, M, K, buf, st); if (rc != QLLM_OK) return rc; a = buf; }
             if (wp) { rc = launch_expand_codes(w, N, K, buf + a_bytes, st); if (rc != QLLM_OK) return rc; w = buf + a_bytes; }
@@ -146,6 +146,7 @@ struct qllm_layer {
     uint8_t *w_codes = nullptr, *codes = nullptr;
     float *w_scale = nullptr, *w_zero = nullptr, *a_scale = nullptr, *a_zero = nullptr;
     void *x_dev = nullptr, *out_dev = nullptr;   // staging for the host-buffer entry point
+    uint8_t* map_image = nullptr;                // reassembly map compiled for the fused kernel (or null)
     std::vector<void*> owned;
 };
 
@@ -170,10 +171,10 @@ int dev_upload(qllm_layer* L, T** p, const T* host, size_t count) {
 
 extern "C" {
 
-int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
-                          const float* ln_beta, float ln_eps, const int32_t* map_ptr,
-                          const int32_t* map_src, const float* map_coef, int bits, uint8_t* codes,
-                          float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream) {
+static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
+                            const float* ln_beta, float ln_eps, const int32_t* map_ptr,
+                            const int32_t* map_src, const float* map_coef, int bits, const void* map_image,
+                            uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream) {
     if (!bits_ok(bits)) return QLLM_ERR_BITS;
     if (!dtype_ok(x_dtype)) return QLLM_ERR_DTYPE;
     if (M < 0 || C <= 0 || C > 49152 || (bits == 4 && (C & 1))) return QLLM_ERR_SHAPE;
@@ -182,8 +183,16 @@ int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const fl
         return QLLM_ERR_NULL;
     if (!aligned16(x) || !aligned16(codes)) return QLLM_ERR_ALIGN;
     return launch_reassemble_quant(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, map_ptr, map_src,
-                                   map_coef, bits, codes, a_scale, a_zero, a_rowsum,
+                                   map_coef, bits, map_image, codes, a_scale, a_zero, a_rowsum,
                                    static_cast<cudaStream_t>(stream));
+}
+
+int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
+                          const float* ln_beta, float ln_eps, const int32_t* map_ptr,
+                          const int32_t* map_src, const float* map_coef, int bits, uint8_t* codes,
+                          float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream) {
+    return reassemble_entry(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, map_ptr, map_src, map_coef, bits,
+                            nullptr, codes, a_scale, a_zero, a_rowsum, stream);
 }
 
 int qllm_calib_absmax(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
@@ -248,6 +257,12 @@ int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const f
     step(dev_upload(L, &L->w_scale, ws, size_t(N)));
     step(dev_upload(L, &L->w_zero, wz, size_t(N)));
     step(dev_upload(L, &L->w_colsum, wcs, size_t(N)));
+    const size_t image_bytes = reassemble_map_image_bytes(C);
+    if (image_bytes) {
+        step(dev_alloc(L, &L->map_image, image_bytes));
+        if (rc == QLLM_OK) step(compile_reassemble_map(C, L->gamma, L->beta, L->ptr, L->src, L->coef, L->map_image, nullptr));
+        if (rc == QLLM_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) rc = QLLM_ERR_CUDA;
+    }
     step(dev_alloc(L, &L->codes, size_t(max_M) * size_t(code_row_bytes(C, a_bits))));
     step(dev_alloc(L, &L->a_scale, size_t(max_M)));
     step(dev_alloc(L, &L->a_zero, size_t(max_M)));
@@ -268,14 +283,25 @@ void qllm_layer_destroy(qllm_layer_t* L) {
     delete L;
 }
 
-int qllm_layer_forward(qllm_layer_t* L, const void* x, int64_t M, void* out, void* stream) {
-    if (!L || !x || !out) return QLLM_ERR_NULL;
+int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void* stream) {
+    if (!L || !x) return QLLM_ERR_NULL;
     if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
-    int rc = qllm_reassemble_quant(x, L->x_dtype, M, L->C, L->gamma, L->beta, L->eps, L->ptr, L->src,
-                                   L->coef, L->a_bits, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream);
-    if (rc != QLLM_OK) return rc;
+    return reassemble_entry(x, L->x_dtype, M, L->C, L->gamma, L->beta, L->eps, L->ptr, L->src, L->coef,
+                            L->a_bits, L->map_image, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream);
+}
+
+int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {
+    if (!L || !out) return QLLM_ERR_NULL;
+    if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
     return qllm_qgemm(L->codes, L->a_scale, L->a_zero, L->w_codes, L->w_scale, L->w_zero, L->w_colsum,
                       L->bias, out, M, L->N, L->C, L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum, stream);
+}
+
+int qllm_layer_forward(qllm_layer_t* L, const void* x, int64_t M, void* out, void* stream) {
+    if (!L || !x || !out) return QLLM_ERR_NULL;
+    int rc = qllm_layer_reassemble_quant(L, x, M, stream);
+    if (rc != QLLM_OK) return rc;
+    return qllm_layer_qgemm(L, M, out, stream);
 }
 
 int qllm_layer_forward_host(qllm_layer_t* L, const void* x_host, int64_t M, void* out_host, void* stream) {

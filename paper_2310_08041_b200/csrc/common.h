@@ -56,9 +56,18 @@ struct EpilogueArgs {
     int raw_acc;            // 1: store int32 accumulators, ignore everything else
 };
 
+// Per-(device, stream) library scratch, grown on demand and never shrunk.
+enum ScratchKind { kScratchExpand = 0, kScratchMapImage = 1, kScratchKinds = 2 };
+int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out);
+
+// The specialised fused kernel consumes a compiled image of the reassembly map (0 bytes: the channel
+// count has no specialised kernel).  map_image = nullptr compiles one per call into stream scratch.
+size_t reassemble_map_image_bytes(int C);
+int compile_reassemble_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
+                           const float* coef, void* image, cudaStream_t st);
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
-                            const float* coef, int bits, uint8_t* codes, float* a_scale,
+                            const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
                             float* a_zero, int32_t* a_rowsum, cudaStream_t st);
 int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                                     const float* beta, float eps, const int32_t* ptr, const int32_t* src,

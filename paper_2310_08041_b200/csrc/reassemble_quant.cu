@@ -23,6 +23,9 @@
 
 #include <cuda_bf16.h>
 
+#include <mutex>
+#include <vector>
+
 #include "common.h"
 #include "device_utils.cuh"
 
@@ -33,6 +36,10 @@ namespace {
 constexpr int kVirt = 256;                     // rows with > 2 entries served through virtual slots
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr int kMagicBits = 0x4B400000;
+
+// Position of channel k in the shared-memory row: even channels in the first half, odd channels in the
+// second, so that the gathers of the even (odd) channels of consecutive pairs walk consecutive banks.
+__device__ __forceinline__ int dpos(int k, int C) { return (k >> 1) + (k & 1) * (C >> 1); }
 
 template <typename XT> struct RowLoad;
 template <> struct RowLoad<__nv_bfloat16> { static constexpr int PER_CHUNK = 8; };
@@ -72,45 +79,47 @@ __device__ __forceinline__ float sum_of(const float* red, int nw4) {
     return s;
 }
 
-template <int CPT, int NTT, typename XT>
-__global__ void __launch_bounds__(NTT ? NTT : 512, (NTT && NTT <= 256) ? 2 : 1)
-reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* __restrict__ gamma,
-                      const float* __restrict__ beta, float eps, const int32_t* __restrict__ ptr,
-                      const int32_t* __restrict__ src, const float* __restrict__ coef, int bits,
-                      uint8_t* __restrict__ codes, float* __restrict__ a_scale, float* __restrict__ a_zero,
-                      int32_t* __restrict__ a_rowsum) {
-    constexpr int PER = RowLoad<XT>::PER_CHUNK;
-    constexpr int NCH = CPT / PER;               // 16-byte chunks of the row per thread
-    constexpr int NP = CPT / 2;                  // channel pairs per thread
-    extern __shared__ __align__(16) uint8_t smem_bytes[];
-    float* red = reinterpret_cast<float*>(smem_bytes);         // [2][4][32] per-warp partials
-    int* redi = reinterpret_cast<int*>(red + 2 * 4 * 32);      // [2][32] code-sum partials
-    int* vrow = redi + 2 * 32;                                 // [kVirt] rows served by virtual slots
-    int* vcount = vrow + kVirt;                                // [4] counter (+ padding)
-    float* d = reinterpret_cast<float*>(vcount + 4);           // [C + kVirt] centred row + virtual slots
+// Compiled form of the reassembly map for one thread layout (CPT channels per thread, NT threads):
+//   rec[slot * NT + t]  = {packed byte offsets of entries 0 and 1 into d, coef0*gamma, coef1*gamma, bias}
+//   tail[t]             = {slots with > 2 entries that did not get a virtual slot (4 bits each, 64 bits), count}
+//   vrow[0..kVirt)      = rows served by virtual slots, nvirt their number
+// Built by one CTA (compile_map_kernel) and loaded by every CTA of the main kernel with coalesced
+// 128-bit loads; the layer object builds it once, direct calls build it per call.
+struct MapImage {
+    uint4* rec;
+    uint4* tail;
+    int* vrow;      // [kVirt + 4]: rows, then nvirt at index kVirt
+};
+__host__ __device__ inline size_t map_image_bytes(int cpt, int nt) {
+    return size_t(cpt) * nt * 16 + size_t(nt) * 16 + size_t(kVirt + 4) * 4;
+}
+__host__ __device__ inline MapImage map_image_at(void* base, int cpt, int nt) {
+    MapImage im;
+    im.rec = static_cast<uint4*>(base);
+    im.tail = im.rec + size_t(cpt) * nt;
+    im.vrow = reinterpret_cast<int*>(im.tail + nt);
+    return im;
+}
 
-    const int t = threadIdx.x, NT = NTT ? NTT : int(blockDim.x), lane = t & 31, warp = t >> 5;
-    const int nw = NT >> 5, nw4 = (nw + 3) & ~3;
-    const bool rot = lane >= 16;
-    const float invC = 1.0f / float(C);
-    const float qmax = float((1 << bits) - 1);
-    const float inv_qmax = 1.0f / qmax;
-
-    for (int i = t; i < 2 * 4 * 32 + 2 * 32 + kVirt + 4; i += NT) red[i] = 0.f;   // zero bit pattern for the int arrays too
-    __syncthreads();
-
-    // ---- map -> registers (once per CTA) ------------------------------------------------
-    uint32_t off[CPT];        // byte offsets into d: entry 0 in the low half, entry 1 in the high half
+// One warp per CTA so that the three rounds of dependent loads of all NT threads run on many SMs at
+// once.  im.vrow[kVirt] (the virtual-slot counter) must be zero at launch; readers clamp it to kVirt.
+template <int CPT>
+__global__ void __launch_bounds__(32)
+compile_map_kernel(int C, int NT, const float* __restrict__ gamma, const float* __restrict__ beta,
+                   const int32_t* __restrict__ ptr, const int32_t* __restrict__ src,
+                   const float* __restrict__ coef, MapImage im) {
+    const int t = blockIdx.x * 32 + threadIdx.x;
+    int* vcount = im.vrow + kVirt;
+    uint32_t off[CPT];
     float cg0[CPT], cg1[CPT], bias[CPT];
-    uint64_t longlist = 0;    // slots (4 bits each) whose row has more than two entries
+    uint64_t longlist = 0;
     int nlong = 0;
     {
-        // three rounds of independent loads (row bounds, entries, gamma/beta) instead of
-        // CPT dependent chains: the set-up is latency-bound and runs once per CTA
+        // three rounds of independent loads (row bounds, entries, gamma/beta) instead of CPT dependent chains
         int j0[CPT], len[CPT];
 #pragma unroll
         for (int slot = 0; slot < CPT; ++slot) {
-            const int c = 2 * (t + NT * (slot >> 1)) + ((slot & 1) ^ int(rot));
+            const int c = 2 * (t + NT * (slot >> 1)) + (slot & 1);
             j0[slot] = __ldg(ptr + c);
             len[slot] = __ldg(ptr + c + 1) - j0[slot];
         }
@@ -132,7 +141,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             float b = 0.f;
             if (beta) b = fmaf(c1[slot], __ldg(beta + s1[slot]), c0[slot] * __ldg(beta + s0[slot]));
             bias[slot] = b;
-            off[slot] = uint32_t(s0[slot] * 4) | (uint32_t(s1[slot] * 4) << 16);
+            off[slot] = uint32_t(dpos(s0[slot], C) * 4) | (uint32_t(dpos(s1[slot], C) * 4) << 16);
         }
 #pragma unroll
         for (int slot = 0; slot < CPT; ++slot) {
@@ -144,7 +153,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
                 // one thread; the owner then reads that slot as its second entry with weight 1.
                 const int vi = atomicAdd(vcount, 1);
                 if (vi < kVirt) {
-                    vrow[vi] = 2 * (t + NT * (slot >> 1)) + ((slot & 1) ^ int(rot));
+                    im.vrow[vi] = 2 * (t + NT * (slot >> 1)) + (slot & 1);
                     cg1[slot] = 1.0f;
                     off[slot] = (off[slot] & 0xFFFFu) | (uint32_t((C + vi) * 4) << 16);
                 } else {                       // more long rows than virtual slots: per-thread tail loop
@@ -154,6 +163,51 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             }
         }
     }
+#pragma unroll
+    for (int slot = 0; slot < CPT; ++slot)
+        im.rec[slot * NT + t] = make_uint4(off[slot], __float_as_uint(cg0[slot]), __float_as_uint(cg1[slot]),
+                                           __float_as_uint(bias[slot]));
+    im.tail[t] = make_uint4(uint32_t(longlist), uint32_t(longlist >> 32), uint32_t(nlong), 0u);
+}
+
+template <int CPT, int NTT, typename XT, bool HAS_BETA, bool FOURBIT>
+__global__ void __launch_bounds__(NTT ? NTT : 512, (NTT && NTT * CPT <= 4096) ? 2 : 1)
+reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* __restrict__ gamma,
+                      float eps, const int32_t* __restrict__ ptr, const int32_t* __restrict__ src,
+                      const float* __restrict__ coef, int bits, MapImage im,
+                      uint8_t* __restrict__ codes, float* __restrict__ a_scale, float* __restrict__ a_zero,
+                      int32_t* __restrict__ a_rowsum) {
+    constexpr int PER = RowLoad<XT>::PER_CHUNK;
+    constexpr int NCH = CPT / PER;               // 16-byte chunks of the row per thread
+    constexpr int NP = CPT / 2;                  // channel pairs per thread
+    extern __shared__ __align__(16) uint8_t smem_bytes[];
+    float* red = reinterpret_cast<float*>(smem_bytes);         // [2][4][32] per-warp partials
+    int* redi = reinterpret_cast<int*>(red + 2 * 4 * 32);      // [2][32] code-sum partials
+    int* vrow = redi + 2 * 32;                                 // [kVirt + 4] rows served by virtual slots, count
+    float* d = reinterpret_cast<float*>(vrow + kVirt + 4);     // [C + kVirt] centred row + virtual slots
+
+    const int t = threadIdx.x, NT = NTT ? NTT : int(blockDim.x), lane = t & 31, warp = t >> 5;
+    const int nw = NT >> 5, nw4 = (nw + 3) & ~3;
+    const float invC = 1.0f / float(C);
+    const float qmax = float((1 << bits) - 1);
+    const float inv_qmax = 1.0f / qmax;
+
+    // ---- compiled map -> registers (once per CTA, coalesced) -----------------------------
+    uint32_t off[CPT];        // byte offsets into d: entry 0 in the low half, entry 1 in the high half
+    float cg0[CPT], cg1[CPT], bias[HAS_BETA ? CPT : 1];
+#pragma unroll
+    for (int slot = 0; slot < CPT; ++slot) {
+        const uint4 r = __ldg(im.rec + slot * NT + t);
+        off[slot] = r.x;
+        cg0[slot] = __uint_as_float(r.y);
+        cg1[slot] = __uint_as_float(r.z);
+        if (HAS_BETA) bias[slot] = __uint_as_float(r.w);
+    }
+    const uint4 tl = __ldg(im.tail + t);
+    const uint64_t longlist = uint64_t(tl.x) | (uint64_t(tl.y) << 32);
+    const int nlong = int(tl.z);
+    for (int i = t; i < 2 * 4 * 32 + 2 * 32; i += NT) red[i] = 0.f;   // zero bit pattern for redi too
+    for (int i = t; i < kVirt + 4; i += NT) vrow[i] = __ldg(im.vrow + i);
 
     // ---- token loop ---------------------------------------------------------------------
     uint4 raw[NCH];
@@ -164,7 +218,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             raw[j] = *reinterpret_cast<const uint4*>(x + m * C + PER * (t + NT * j));
     }
     __syncthreads();
-    const int nvirt = min(*vcount, kVirt);
+    const int nvirt = min(vrow[kVirt], kVirt);
     int par = 0;
     int64_t m_prev = -1;
     for (; m < M; m += gridDim.x, par ^= 1) {
@@ -216,11 +270,17 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
         }
 #pragma unroll
         for (int j = 0; j < NCH; ++j) {
-            float* dst = d + PER * (t + NT * j);
-#pragma unroll
-            for (int k = 0; k < PER; k += 4)
-                *reinterpret_cast<float4*>(dst + k) =
-                    make_float4(xv[PER * j + k], xv[PER * j + k + 1], xv[PER * j + k + 2], xv[PER * j + k + 3]);
+            // channels PER*u .. PER*u + PER-1: even ones to d[PER/2 * u ..], odd ones to d[C/2 + PER/2 * u ..]
+            const int u = t + NT * j;
+            float* ev = d + (PER / 2) * u;
+            float* od = ev + (C >> 1);
+            if constexpr (PER == 8) {
+                *reinterpret_cast<float4*>(ev) = make_float4(xv[8 * j], xv[8 * j + 2], xv[8 * j + 4], xv[8 * j + 6]);
+                *reinterpret_cast<float4*>(od) = make_float4(xv[8 * j + 1], xv[8 * j + 3], xv[8 * j + 5], xv[8 * j + 7]);
+            } else {
+                *reinterpret_cast<float2*>(ev) = make_float2(xv[4 * j], xv[4 * j + 2]);
+                *reinterpret_cast<float2*>(od) = make_float2(xv[4 * j + 1], xv[4 * j + 3]);
+            }
         }
         sq = warp_sum(sq);
         if (lane == 0) rsq[warp] = sq;
@@ -234,7 +294,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
                 float e = 0.f;
                 for (int j = __ldg(ptr + c) + 1; j < __ldg(ptr + c + 1); ++j) {
                     const int sj = __ldg(src + j);
-                    e = fmaf(__ldg(coef + j) * __ldg(gamma + sj), d[sj], e);
+                    e = fmaf(__ldg(coef + j) * __ldg(gamma + sj), d[dpos(sj, C)], e);
                 }
                 d[C + vi] = e;
             }
@@ -252,11 +312,11 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
         }
         for (int k = 0; k < nlong; ++k) {                              // rows with > 2 entries (rare)
             const int slot = int((longlist >> (4 * k)) & 15u);
-            const int c = 2 * (t + NT * (slot >> 1)) + ((slot & 1) ^ int(rot));
+            const int c = 2 * (t + NT * (slot >> 1)) + (slot & 1);
             float e = 0.f;
             for (int j = ptr[c] + 2; j < ptr[c + 1]; ++j) {
                 const int sj = src[j];
-                e = fmaf(coef[j] * gamma[sj], d[sj], e);
+                e = fmaf(coef[j] * gamma[sj], d[dpos(sj, C)], e);
             }
 #pragma unroll
             for (int q = 0; q < CPT; ++q)
@@ -265,7 +325,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
         float lo = INFINITY, hi = -INFINITY;
 #pragma unroll
         for (int slot = 0; slot < CPT; ++slot) {
-            v[slot] = fmaf(rstd, v[slot], bias[slot]);
+            v[slot] = HAS_BETA ? fmaf(rstd, v[slot], bias[slot]) : rstd * v[slot];
             lo = fminf(lo, v[slot]);
             hi = fmaxf(hi, v[slot]);
         }
@@ -305,17 +365,15 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             }
         }
         int csum = 0;
-        if (bits == 4) {
-            // one byte per pair: low nibble = even channel.  Pack as held, then swap the nibbles
-            // on the lanes that keep their pairs swapped.
+        if (FOURBIT) {
+            // one byte per pair: low nibble = even channel
             uint32_t w[NP / 4];
 #pragma unroll
             for (int g = 0; g < NP / 4; ++g) {
                 uint32_t p = 0;
 #pragma unroll
                 for (int i = 3; i >= 0; --i) p = pack_sat_u4(n[2 * (4 * g + i) + 1], n[2 * (4 * g + i)], p);
-                const uint32_t sw = ((p << 4) & 0xF0F0F0F0u) | ((p >> 4) & 0x0F0F0F0Fu);
-                w[g] = rot ? sw : p;
+                w[g] = p;
                 const uint32_t nib = (p & 0x0F0F0F0Fu) + ((p >> 4) & 0x0F0F0F0Fu);
                 csum = int(__dp4a(nib, 0x01010101u, uint32_t(csum)));
             }
@@ -327,8 +385,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             uint16_t* out = reinterpret_cast<uint16_t*>(codes + m * C) + t;
 #pragma unroll
             for (int i = 0; i < NP; ++i) {
-                const int e = rot ? n[2 * i + 1] : n[2 * i];
-                const int o = rot ? n[2 * i] : n[2 * i + 1];
+                const int e = n[2 * i], o = n[2 * i + 1];
                 const uint32_t p = pack_sat_u8(min(o, top), min(e, top), 0);
                 out[NT * i] = uint16_t(p);
                 csum += int(p & 0xFFu) + int(p >> 8);
@@ -359,11 +416,11 @@ int sm_count() {
     return n;
 }
 
-template <int CPT, int NTT, typename XT>
-int launch_fast(const void* x, int64_t M, int C, const float* gamma, const float* beta, float eps,
-                const int32_t* ptr, const int32_t* src, const float* coef, int bits, uint8_t* codes,
+template <int CPT, int NTT, typename XT, bool HAS_BETA, bool FOURBIT>
+int launch_main(const void* x, int64_t M, int C, const float* gamma, float eps, const int32_t* ptr,
+                const int32_t* src, const float* coef, int bits, const MapImage& im, uint8_t* codes,
                 float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
-    auto kern = reassemble_quant_fast<CPT, NTT, XT>;
+    auto kern = reassemble_quant_fast<CPT, NTT, XT, HAS_BETA, FOURBIT>;
     const int nt = C / CPT;
     const size_t smem = size_t(C + kVirt) * 4 + (2 * 4 * 32 + 2 * 32 + kVirt + 4) * 4;
     if (smem > 48 * 1024)
@@ -372,30 +429,77 @@ int launch_fast(const void* x, int64_t M, int C, const float* gamma, const float
     QLLM_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, nt, smem));
     if (per_sm < 1) per_sm = 1;
     const int grid = int(std::min<int64_t>(M, int64_t(sm_count()) * per_sm));
-    kern<<<grid, nt, smem, st>>>(static_cast<const XT*>(x), M, C, gamma, beta, eps, ptr, src, coef, bits,
-                                 codes, a_scale, a_zero, a_rowsum);
+    kern<<<grid, nt, smem, st>>>(static_cast<const XT*>(x), M, C, gamma, eps, ptr, src, coef, bits, im, codes,
+                                 a_scale, a_zero, a_rowsum);
     return after_launch();
+}
+
+template <int CPT, int NTT, typename XT>
+int launch_layout(const void* x, int64_t M, int C, const float* gamma, bool has_beta, float eps,
+                  const int32_t* ptr, const int32_t* src, const float* coef, int bits, const MapImage& im,
+                  uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
+#define QLLM_MAIN(B, F) launch_main<CPT, NTT, XT, B, F>(x, M, C, gamma, eps, ptr, src, coef, bits, im, codes, a_scale, a_zero, a_rowsum, st)
+    // run-time thread counts keep one variant per bit packing (the bias registers are always present)
+    if (NTT == 0 || has_beta) return bits == 4 ? QLLM_MAIN(true, true) : QLLM_MAIN(true, false);
+    return bits == 4 ? QLLM_MAIN(false, true) : QLLM_MAIN(false, false);
+#undef QLLM_MAIN
+}
+
+// Thread layout of the specialised kernel for a channel count: channels per thread (0 = none).
+int layout_cpt(int C) {
+    if (C % 512 == 0 && C <= 8192) return 16;
+    if (C % 256 == 0 && C <= 4096) return 8;
+    return 0;
 }
 
 }  // namespace
 
-#define QLLM_RQ_ARGS x, M, C, gamma, beta, eps, ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, st
+size_t reassemble_map_image_bytes(int C) {
+    const int cpt = layout_cpt(C);
+    return cpt ? map_image_bytes(cpt, C / cpt) : 0;
+}
+
+int compile_reassemble_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
+                           const float* coef, void* image, cudaStream_t st) {
+    const int cpt = layout_cpt(C);
+    if (!cpt) return QLLM_ERR_UNSUPPORTED;
+    const int nt = C / cpt;
+    const MapImage im = map_image_at(image, cpt, nt);
+    QLLM_CUDA_TRY(cudaMemsetAsync(im.vrow + kVirt, 0, sizeof(int), st));
+    if (cpt == 16) compile_map_kernel<16><<<nt / 32, 32, 0, st>>>(C, nt, gamma, beta, ptr, src, coef, im);
+    else compile_map_kernel<8><<<nt / 32, 32, 0, st>>>(C, nt, gamma, beta, ptr, src, coef, im);
+    return after_launch();
+}
 
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
-                            const float* coef, int bits, uint8_t* codes, float* a_scale,
+                            const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
                             float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
-    const bool bf = x_dtype == QLLM_BF16;
+    const int cpt = layout_cpt(C);
+    if (!cpt)
+        return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
+                                               a_scale, a_zero, a_rowsum, st);
+    const int nt = C / cpt;
+    if (!map_image) {
+        // direct call: compile the map for this launch into per-stream library scratch
+        uint8_t* buf = nullptr;
+        int rc = stream_scratch(kScratchMapImage, st, map_image_bytes(cpt, nt), &buf);
+        if (rc != QLLM_OK) return rc;
+        rc = compile_reassemble_map(C, gamma, beta, ptr, src, coef, buf, st);
+        if (rc != QLLM_OK) return rc;
+        map_image = buf;
+    }
+    const MapImage im = map_image_at(const_cast<void*>(map_image), cpt, nt);
+    const bool bf = x_dtype == QLLM_BF16, hb = beta != nullptr;
+#define QLLM_RQ_ARGS x, M, C, gamma, hb, eps, ptr, src, coef, bits, im, codes, a_scale, a_zero, a_rowsum, st
     // LLaMA hidden sizes get compile-time thread counts (immediate offsets, unrolled reductions)
-    if (bf && C == 4096) return launch_fast<16, 256, __nv_bfloat16>(QLLM_RQ_ARGS);
-    if (bf && C == 5120) return launch_fast<16, 320, __nv_bfloat16>(QLLM_RQ_ARGS);
-    if (bf && C == 8192) return launch_fast<16, 512, __nv_bfloat16>(QLLM_RQ_ARGS);
-    if (C % 512 == 0 && C <= 8192)
-        return bf ? launch_fast<16, 0, __nv_bfloat16>(QLLM_RQ_ARGS) : launch_fast<16, 0, float>(QLLM_RQ_ARGS);
-    if (C % 256 == 0 && C <= 4096)
-        return bf ? launch_fast<8, 0, __nv_bfloat16>(QLLM_RQ_ARGS) : launch_fast<8, 0, float>(QLLM_RQ_ARGS);
-    return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
-                                           a_scale, a_zero, a_rowsum, st);
+    if (bf && C == 4096) return launch_layout<16, 256, __nv_bfloat16>(QLLM_RQ_ARGS);
+    if (bf && C == 5120) return launch_layout<16, 320, __nv_bfloat16>(QLLM_RQ_ARGS);
+    if (bf && C == 8192) return launch_layout<16, 512, __nv_bfloat16>(QLLM_RQ_ARGS);
+    if (cpt == 16)
+        return bf ? launch_layout<16, 0, __nv_bfloat16>(QLLM_RQ_ARGS) : launch_layout<16, 0, float>(QLLM_RQ_ARGS);
+    return bf ? launch_layout<8, 0, __nv_bfloat16>(QLLM_RQ_ARGS) : launch_layout<8, 0, float>(QLLM_RQ_ARGS);
+#undef QLLM_RQ_ARGS
 }
 
 }  // namespace qllm
