@@ -33,7 +33,8 @@ namespace qllm {
 
 namespace {
 
-constexpr int kVirt = 256;                     // rows with > 2 entries served through virtual slots
+constexpr int kVirt = 2048;                    // virtual slots (rows with more than one entry)
+constexpr int kVirtEntries = 4;                // entries a virtual-slot record can hold
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
 constexpr int kMagicBits = 0x4B400000;
 
@@ -53,6 +54,16 @@ __device__ __forceinline__ float redux_min(float v) {
 __device__ __forceinline__ float redux_max(float v) {
     float r;
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float r;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
 // d = sat_u4(a) << 4 | sat_u4(b) | c << 8
@@ -80,98 +91,85 @@ __device__ __forceinline__ float sum_of(const float* red, int nw4) {
 }
 
 // Compiled form of the reassembly map for one thread layout (CPT channels per thread, NT threads):
-//   rec[slot * NT + t]  = {packed byte offsets of entries 0 and 1 into d, coef0*gamma, coef1*gamma, bias}
-//   tail[t]             = {slots with > 2 entries that did not get a virtual slot (4 bits each, 64 bits), count}
-//   vrow[0..kVirt)      = rows served by virtual slots, nvirt their number
-// Built by one CTA (compile_map_kernel) and loaded by every CTA of the main kernel with coalesced
-// 128-bit loads; the layer object builds it once, direct calls build it per call.
+//   rec[slot * NT + t] = {byte offset into d, weight, bias, flags}  flags bit 0: the row takes the
+//                        per-thread CSR fallback (entries 1.. are added from the raw map)
+//   vrec[2 vi], [2 vi + 1] = virtual slot vi: {offsets 0|1, offsets 2|3, w0, w1}, {w2, w3, n, 0}
+//   head[0] = virtual slots handed out (a counter; readers clamp it to kVirt)
+// Built by compile_map_kernel and loaded by the main kernel with coalesced 128-bit loads; the layer
+// object builds it once, direct calls build it per call.
 struct MapImage {
     uint4* rec;
-    uint4* tail;
-    int* vrow;      // [kVirt + 4]: rows, then nvirt at index kVirt
+    uint4* vrec;
+    int* head;
 };
 __host__ __device__ inline size_t map_image_bytes(int cpt, int nt) {
-    return size_t(cpt) * nt * 16 + size_t(nt) * 16 + size_t(kVirt + 4) * 4;
+    return size_t(cpt) * nt * 16 + size_t(kVirt) * 32 + 16;
 }
 __host__ __device__ inline MapImage map_image_at(void* base, int cpt, int nt) {
     MapImage im;
     im.rec = static_cast<uint4*>(base);
-    im.tail = im.rec + size_t(cpt) * nt;
-    im.vrow = reinterpret_cast<int*>(im.tail + nt);
+    im.vrec = im.rec + size_t(cpt) * nt;
+    im.head = reinterpret_cast<int*>(im.vrec + 2 * size_t(kVirt));
     return im;
 }
 
-// One warp per CTA so that the three rounds of dependent loads of all NT threads run on many SMs at
-// once.  im.vrow[kVirt] (the virtual-slot counter) must be zero at launch; readers clamp it to kVirt.
+// One warp per CTA so that the dependent load rounds of all NT threads run on many SMs at once.
+// im.head[0] must be zero at launch.
 template <int CPT>
 __global__ void __launch_bounds__(32)
 compile_map_kernel(int C, int NT, const float* __restrict__ gamma, const float* __restrict__ beta,
                    const int32_t* __restrict__ ptr, const int32_t* __restrict__ src,
                    const float* __restrict__ coef, MapImage im) {
     const int t = blockIdx.x * 32 + threadIdx.x;
-    int* vcount = im.vrow + kVirt;
-    uint32_t off[CPT];
-    float cg0[CPT], cg1[CPT], bias[CPT];
-    uint64_t longlist = 0;
-    int nlong = 0;
-    {
-        // three rounds of independent loads (row bounds, entries, gamma/beta) instead of CPT dependent chains
-        int j0[CPT], len[CPT];
+    int j0[CPT], len[CPT];
 #pragma unroll
-        for (int slot = 0; slot < CPT; ++slot) {
-            const int c = 2 * (t + NT * (slot >> 1)) + (slot & 1);
-            j0[slot] = __ldg(ptr + c);
-            len[slot] = __ldg(ptr + c + 1) - j0[slot];
-        }
-        int s0[CPT], s1[CPT];
-        float c0[CPT], c1[CPT];
+    for (int slot = 0; slot < CPT; ++slot) {
+        const int c = 2 * (t + NT * (slot >> 1)) + (slot & 1);
+        j0[slot] = __ldg(ptr + c);
+        len[slot] = __ldg(ptr + c + 1) - j0[slot];
+    }
+    int s0[CPT];
+    float c0[CPT];
 #pragma unroll
-        for (int slot = 0; slot < CPT; ++slot) {
-            const int j1 = j0[slot] + (len[slot] >= 2 ? 1 : 0);
-            s0[slot] = __ldg(src + j0[slot]);
-            s1[slot] = __ldg(src + j1);
-            c0[slot] = __ldg(coef + j0[slot]);
-            c1[slot] = __ldg(coef + j1);
-        }
-#pragma unroll
-        for (int slot = 0; slot < CPT; ++slot) {
-            if (len[slot] < 2) c1[slot] = 0.f;
-            cg0[slot] = c0[slot] * __ldg(gamma + s0[slot]);
-            cg1[slot] = c1[slot] * __ldg(gamma + s1[slot]);
-            float b = 0.f;
-            if (beta) b = fmaf(c1[slot], __ldg(beta + s1[slot]), c0[slot] * __ldg(beta + s0[slot]));
-            bias[slot] = b;
-            off[slot] = uint32_t(dpos(s0[slot], C) * 4) | (uint32_t(dpos(s1[slot], C) * 4) << 16);
-        }
-#pragma unroll
-        for (int slot = 0; slot < CPT; ++slot) {
-            if (len[slot] > 2) {
-                if (beta)
-                    for (int j = j0[slot] + 2; j < j0[slot] + len[slot]; ++j)
-                        bias[slot] = fmaf(coef[j], beta[src[j]], bias[slot]);
-                // Entries 1.. of this row are summed once per token into virtual slot d[C + vi] by
-                // one thread; the owner then reads that slot as its second entry with weight 1.
-                const int vi = atomicAdd(vcount, 1);
-                if (vi < kVirt) {
-                    im.vrow[vi] = 2 * (t + NT * (slot >> 1)) + (slot & 1);
-                    cg1[slot] = 1.0f;
-                    off[slot] = (off[slot] & 0xFFFFu) | (uint32_t((C + vi) * 4) << 16);
-                } else {                       // more long rows than virtual slots: per-thread tail loop
-                    longlist |= uint64_t(slot) << (4 * nlong);
-                    ++nlong;
-                }
-            }
-        }
+    for (int slot = 0; slot < CPT; ++slot) {
+        s0[slot] = __ldg(src + j0[slot]);
+        c0[slot] = __ldg(coef + j0[slot]);
     }
 #pragma unroll
-    for (int slot = 0; slot < CPT; ++slot)
-        im.rec[slot * NT + t] = make_uint4(off[slot], __float_as_uint(cg0[slot]), __float_as_uint(cg1[slot]),
-                                           __float_as_uint(bias[slot]));
-    im.tail[t] = make_uint4(uint32_t(longlist), uint32_t(longlist >> 32), uint32_t(nlong), 0u);
+    for (int slot = 0; slot < CPT; ++slot) {
+        uint32_t off = uint32_t(dpos(s0[slot], C) * 4);
+        float w = c0[slot] * __ldg(gamma + s0[slot]);
+        float b = beta ? c0[slot] * __ldg(beta + s0[slot]) : 0.f;
+        uint32_t flags = 0;
+        const int n = len[slot];
+        if (n > 1) {                                  // merged row (short loops, minority of rows)
+            if (beta)
+                for (int j = j0[slot] + 1; j < j0[slot] + n; ++j)
+                    b = fmaf(__ldg(coef + j), __ldg(beta + __ldg(src + j)), b);
+            const int vi = n <= kVirtEntries ? atomicAdd(im.head, 1) : kVirt;
+            if (vi < kVirt) {
+                uint32_t o[kVirtEntries] = {0, 0, 0, 0};
+                float ww[kVirtEntries] = {0.f, 0.f, 0.f, 0.f};
+                for (int e = 0; e < n; ++e) {
+                    const int sj = __ldg(src + j0[slot] + e);
+                    o[e] = uint32_t(dpos(sj, C) * 4);
+                    ww[e] = __ldg(coef + j0[slot] + e) * __ldg(gamma + sj);
+                }
+                im.vrec[2 * vi] = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), __float_as_uint(ww[0]),
+                                             __float_as_uint(ww[1]));
+                im.vrec[2 * vi + 1] = make_uint4(__float_as_uint(ww[2]), __float_as_uint(ww[3]), uint32_t(n), 0u);
+                off = uint32_t((C + vi) * 4);
+                w = 1.0f;
+            } else {
+                flags = 1;                            // first entry in registers, the rest from the CSR
+            }
+        }
+        im.rec[slot * NT + t] = make_uint4(off, __float_as_uint(w), __float_as_uint(b), flags);
+    }
 }
 
 template <int CPT, int NTT, typename XT, bool HAS_BETA, bool FOURBIT>
-__global__ void __launch_bounds__(NTT ? NTT : 512, (NTT && NTT * CPT <= 4096) ? 2 : 1)
+__global__ void __launch_bounds__(NTT ? NTT : 512, (NTT && NTT <= 256) ? 3 : 1)
 reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* __restrict__ gamma,
                       float eps, const int32_t* __restrict__ ptr, const int32_t* __restrict__ src,
                       const float* __restrict__ coef, int bits, MapImage im,
@@ -183,8 +181,7 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
     extern __shared__ __align__(16) uint8_t smem_bytes[];
     float* red = reinterpret_cast<float*>(smem_bytes);         // [2][4][32] per-warp partials
     int* redi = reinterpret_cast<int*>(red + 2 * 4 * 32);      // [2][32] code-sum partials
-    int* vrow = redi + 2 * 32;                                 // [kVirt + 4] rows served by virtual slots, count
-    float* d = reinterpret_cast<float*>(vrow + kVirt + 4);     // [C + kVirt] centred row + virtual slots
+    float* d = reinterpret_cast<float*>(redi + 2 * 32);        // [C + kVirt] centred row + virtual slots
 
     const int t = threadIdx.x, NT = NTT ? NTT : int(blockDim.x), lane = t & 31, warp = t >> 5;
     const int nw = NT >> 5, nw4 = (nw + 3) & ~3;
@@ -193,21 +190,20 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
     const float inv_qmax = 1.0f / qmax;
 
     // ---- compiled map -> registers (once per CTA, coalesced) -----------------------------
-    uint32_t off[CPT];        // byte offsets into d: entry 0 in the low half, entry 1 in the high half
-    float cg0[CPT], cg1[CPT], bias[HAS_BETA ? CPT : 1];
+    uint32_t off[CPT];
+    float wgt[CPT], bias[HAS_BETA ? CPT : 1];
+    uint32_t fallback = 0;                       // bit per slot: the row continues in the raw CSR
 #pragma unroll
     for (int slot = 0; slot < CPT; ++slot) {
         const uint4 r = __ldg(im.rec + slot * NT + t);
         off[slot] = r.x;
-        cg0[slot] = __uint_as_float(r.y);
-        cg1[slot] = __uint_as_float(r.z);
-        if (HAS_BETA) bias[slot] = __uint_as_float(r.w);
+        wgt[slot] = __uint_as_float(r.y);
+        if (HAS_BETA) bias[slot] = __uint_as_float(r.z);
+        fallback |= (r.w & 1u) << slot;
     }
-    const uint4 tl = __ldg(im.tail + t);
-    const uint64_t longlist = uint64_t(tl.x) | (uint64_t(tl.y) << 32);
-    const int nlong = int(tl.z);
+    const int nvirt = min(__ldg(im.head), kVirt);
     for (int i = t; i < 2 * 4 * 32 + 2 * 32; i += NT) red[i] = 0.f;   // zero bit pattern for redi too
-    for (int i = t; i < kVirt + 4; i += NT) vrow[i] = __ldg(im.vrow + i);
+    const char* dbytes = reinterpret_cast<const char*>(d);
 
     // ---- token loop ---------------------------------------------------------------------
     uint4 raw[NCH];
@@ -218,7 +214,6 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             raw[j] = *reinterpret_cast<const uint4*>(x + m * C + PER * (t + NT * j));
     }
     __syncthreads();
-    const int nvirt = min(vrow[kVirt], kVirt);
     int par = 0;
     int64_t m_prev = -1;
     for (; m < M; m += gridDim.x, par ^= 1) {
@@ -288,46 +283,47 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
         const float var = sum_of(rsq, nw4) * invC;
         const float rstd = rsqrtf(var + eps);        // a common factor of the whole row: its last-bit
                                                      // error rescales alpha with the row, codes unchanged
+        // -- merged rows: one thread per row sums its entries into the row's virtual slot
         if (nvirt > 0) {                             // uniform over the CTA
             for (int vi = t; vi < nvirt; vi += NT) {
-                const int c = vrow[vi];
-                float e = 0.f;
-                for (int j = __ldg(ptr + c) + 1; j < __ldg(ptr + c + 1); ++j) {
-                    const int sj = __ldg(src + j);
-                    e = fmaf(__ldg(coef + j) * __ldg(gamma + sj), d[dpos(sj, C)], e);
+                const uint4 r0 = __ldg(im.vrec + 2 * vi), r1 = __ldg(im.vrec + 2 * vi + 1);
+                float e = __uint_as_float(r0.z) * *reinterpret_cast<const float*>(dbytes + (r0.x & 0xFFFFu));
+                e = fmaf(__uint_as_float(r0.w), *reinterpret_cast<const float*>(dbytes + (r0.x >> 16)), e);
+                if (r1.z > 2u) {
+                    e = fmaf(__uint_as_float(r1.x), *reinterpret_cast<const float*>(dbytes + (r0.y & 0xFFFFu)), e);
+                    if (r1.z > 3u)
+                        e = fmaf(__uint_as_float(r1.y), *reinterpret_cast<const float*>(dbytes + (r0.y >> 16)), e);
                 }
                 d[C + vi] = e;
             }
             __syncthreads();                                           // S2b
         }
-        // -- reassembly: gather from d with the register-resident map
-        const char* dbytes = reinterpret_cast<const char*>(d);
+        // -- reassembly: one gather per channel with the register-resident map
         float v[CPT];
 #pragma unroll
-        for (int slot = 0; slot < CPT; ++slot) {
-            const float a0 = *reinterpret_cast<const float*>(dbytes + (off[slot] & 0xFFFFu));
-            const float a1 = *reinterpret_cast<const float*>(dbytes + (off[slot] >> 16));
-            const float acc = fmaf(cg1[slot], a1, cg0[slot] * a0);
-            v[slot] = acc;
-        }
-        for (int k = 0; k < nlong; ++k) {                              // rows with > 2 entries (rare)
-            const int slot = int((longlist >> (4 * k)) & 15u);
-            const int c = 2 * (t + NT * (slot >> 1)) + (slot & 1);
-            float e = 0.f;
-            for (int j = ptr[c] + 2; j < ptr[c + 1]; ++j) {
-                const int sj = src[j];
-                e = fmaf(coef[j] * gamma[sj], d[dpos(sj, C)], e);
-            }
+        for (int slot = 0; slot < CPT; ++slot)
+            v[slot] = wgt[slot] * *reinterpret_cast<const float*>(dbytes + off[slot]);
+        if (fallback) {                                                // rows beyond the virtual slots (rare)
+            for (uint32_t fb = fallback; fb; fb &= fb - 1) {
+                const int slot = __ffs(int(fb)) - 1;
+                const int c = 2 * (t + NT * (slot >> 1)) + (slot & 1);
+                float e = 0.f;
+                for (int j = ptr[c] + 1; j < ptr[c + 1]; ++j) {
+                    const int sj = src[j];
+                    e = fmaf(coef[j] * gamma[sj], d[dpos(sj, C)], e);
+                }
 #pragma unroll
-            for (int q = 0; q < CPT; ++q)
-                if (q == slot) v[q] += e;
+                for (int q = 0; q < CPT; ++q)
+                    if (q == slot) v[q] += e;
+            }
         }
         float lo = INFINITY, hi = -INFINITY;
 #pragma unroll
-        for (int slot = 0; slot < CPT; ++slot) {
+        for (int slot = 0; slot < CPT; slot += 2) {
             v[slot] = HAS_BETA ? fmaf(rstd, v[slot], bias[slot]) : rstd * v[slot];
-            lo = fminf(lo, v[slot]);
-            hi = fmaxf(hi, v[slot]);
+            v[slot + 1] = HAS_BETA ? fmaf(rstd, v[slot + 1], bias[slot + 1]) : rstd * v[slot + 1];
+            lo = min3(lo, v[slot], v[slot + 1]);
+            hi = max3(hi, v[slot], v[slot + 1]);
         }
         lo = redux_min(lo);
         hi = redux_max(hi);
@@ -337,8 +333,8 @@ reassemble_quant_fast(const XT* __restrict__ x, int64_t M, int C, const float* _
             const float4 a = *reinterpret_cast<const float4*>(rlo + w);
             const float4 b = *reinterpret_cast<const float4*>(rhi + w);
             if (w + 3 < nw) {
-                lo = fminf(fminf(lo, fminf(a.x, a.y)), fminf(a.z, a.w));
-                hi = fmaxf(fmaxf(hi, fmaxf(b.x, b.y)), fmaxf(b.z, b.w));
+                lo = min3(min3(lo, a.x, a.y), a.z, a.w);
+                hi = max3(max3(hi, b.x, b.y), b.z, b.w);
             } else {
                 lo = fminf(lo, a.x); hi = fmaxf(hi, b.x);
                 if (w + 1 < nw) { lo = fminf(lo, a.y); hi = fmaxf(hi, b.y); }
@@ -422,7 +418,7 @@ int launch_main(const void* x, int64_t M, int C, const float* gamma, float eps, 
                 float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
     auto kern = reassemble_quant_fast<CPT, NTT, XT, HAS_BETA, FOURBIT>;
     const int nt = C / CPT;
-    const size_t smem = size_t(C + kVirt) * 4 + (2 * 4 * 32 + 2 * 32 + kVirt + 4) * 4;
+    const size_t smem = size_t(C + kVirt) * 4 + (2 * 4 * 32 + 2 * 32) * 4;
     if (smem > 48 * 1024)
         QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     int per_sm = 0;
@@ -465,7 +461,7 @@ int compile_reassemble_map(int C, const float* gamma, const float* beta, const i
     if (!cpt) return QLLM_ERR_UNSUPPORTED;
     const int nt = C / cpt;
     const MapImage im = map_image_at(image, cpt, nt);
-    QLLM_CUDA_TRY(cudaMemsetAsync(im.vrow + kVirt, 0, sizeof(int), st));
+    QLLM_CUDA_TRY(cudaMemsetAsync(im.head, 0, 16, st));
     if (cpt == 16) compile_map_kernel<16><<<nt / 32, 32, 0, st>>>(C, nt, gamma, beta, ptr, src, coef, im);
     else compile_map_kernel<8><<<nt / 32, 32, 0, st>>>(C, nt, gamma, beta, ptr, src, coef, im);
     return after_launch();
