@@ -85,8 +85,14 @@ int check_gemm_shape(int64_t M, int N, int K, int a_bits, int w_bits) {
 // shared memory, which caps the tensor pipe near 40 %.
 constexpr int64_t kExpandMinM = 512;
 
+bool expand_path(int64_t M, int N, int K, int a_bits, int w_bits) {
+    return M > 16 && M >= kExpandMinM && (a_bits == 4 || w_bits == 4) && qgemm_tc_supported(M, N, K, a_bits, w_bits);
+}
+
+// w_ready: the weight codes already expanded to bytes at the weight slot of this stream's expand scratch
+// (done ahead of time on another stream by the layer object), or nullptr.
 int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
-                  const EpilogueArgs& ep, cudaStream_t st, bool may_allocate) {
+                  const EpilogueArgs& ep, cudaStream_t st, bool may_allocate, const uint8_t* w_ready = nullptr) {
     if (M == 0) return QLLM_OK;
     if (M <= 16 && qgemm_decode_supported(M, N, K, a_bits, w_bits))
         return launch_qgemm_decode(a, w, M, N, K, a_bits, w_bits, ep, st);
@@ -98,7 +104,8 @@ int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, i
             int rc = stream_scratch(kScratchExpand, st, a_bytes + w_bytes, &buf);
             if (rc != QLLM_OK) return rc;
             if (ap) { rc = launch_expand_codes(a, M, K, buf, st); if (rc != QLLM_OK) return rc; a = buf; }
-            if (wp) { rc = launch_expand_codes(w, N, K, buf + a_bytes, st); if (rc != QLLM_OK) return rc; w = buf + a_bytes; }
+            if (wp && w_ready == buf + a_bytes) w = w_ready;
+            else if (wp) { rc = launch_expand_codes(w, N, K, buf + a_bytes, st); if (rc != QLLM_OK) return rc; w = buf + a_bytes; }
             return launch_qgemm_tc(a, w, M, N, K, 8, 8, ep, st);
         }
         return launch_qgemm_tc(a, w, M, N, K, a_bits, w_bits, ep, st);
@@ -111,7 +118,7 @@ int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, i
 int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
                const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
                int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
-               cudaStream_t st, bool may_allocate) {
+               cudaStream_t st, bool may_allocate, const uint8_t* w_ready) {
     int rc = check_gemm_shape(M, N, K, a_bits, w_bits);
     if (rc != QLLM_OK) return rc;
     if (!dtype_ok(out_dtype)) return QLLM_ERR_DTYPE;
@@ -129,7 +136,7 @@ int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, 
         a_rowsum = scratch;
     }
     EpilogueArgs ep{a_scale, a_zero, a_rowsum, w_scale, w_zero, w_colsum, bias, out, out_dtype, 0};
-    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, st, may_allocate);
+    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, st, may_allocate, w_ready);
 }
 
 }  // namespace qllm
@@ -147,6 +154,12 @@ struct qllm_layer {
     float *w_scale = nullptr, *w_zero = nullptr, *a_scale = nullptr, *a_zero = nullptr;
     void *x_dev = nullptr, *out_dev = nullptr;   // staging for the host-buffer entry point
     uint8_t* map_image = nullptr;                // reassembly map compiled for the fused kernel (or null)
+    // The byte expansion of the 4-bit weights that a large-M GEMM needs does not depend on the tokens, so the
+    // pre-GEMM call starts it on a side stream; the GEMM call joins it.
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    const uint8_t* w_ready = nullptr;            // expanded weights in flight / ready for the next GEMM call
+    int64_t w_ready_M = -1;
     std::vector<void*> owned;
 };
 
@@ -211,7 +224,7 @@ int qllm_qgemm(const uint8_t* codes, const float* a_scale, const float* a_zero, 
                void* out, int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype,
                const int32_t* a_rowsum, void* stream) {
     return gemm_entry(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, bias, out, M, N, K, a_bits,
-                      w_bits, out_dtype, a_rowsum, static_cast<cudaStream_t>(stream), true);
+                      w_bits, out_dtype, a_rowsum, static_cast<cudaStream_t>(stream), true, nullptr);
 }
 
 int qllm_qgemm_acc(const uint8_t* codes, const uint8_t* w_codes, int32_t* acc, int64_t M, int N, int K,
@@ -272,6 +285,12 @@ int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const f
     step(dev_alloc(L, &xd, size_t(max_M) * size_t(C) * xb));
     step(dev_alloc(L, &od, size_t(max_M) * size_t(N) * ob));
     L->x_dev = xd; L->out_dev = od;
+    if (rc == QLLM_OK && w_bits == 4) {
+        if (cudaStreamCreateWithFlags(&L->side, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&L->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming) != cudaSuccess)
+            rc = cuda_fail(cudaGetLastError());
+    }
     if (rc != QLLM_OK) { qllm_layer_destroy(L); return rc; }
     *out = L;
     return QLLM_OK;
@@ -279,6 +298,9 @@ int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const f
 
 void qllm_layer_destroy(qllm_layer_t* L) {
     if (!L) return;
+    if (L->side) { cudaStreamSynchronize(L->side); cudaStreamDestroy(L->side); }
+    if (L->ev_fork) cudaEventDestroy(L->ev_fork);
+    if (L->ev_join) cudaEventDestroy(L->ev_join);
     for (void* p : L->owned) cudaFree(p);
     delete L;
 }
@@ -286,6 +308,22 @@ void qllm_layer_destroy(qllm_layer_t* L) {
 int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void* stream) {
     if (!L || !x) return QLLM_ERR_NULL;
     if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
+    L->w_ready = nullptr;
+    if (L->side && expand_path(M, L->N, L->C, L->a_bits, L->w_bits)) {
+        // start expanding the weights for the coming GEMM on the side stream: it is independent of the tokens
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        const size_t a_bytes = L->a_bits == 4 ? size_t(M) * L->C : 0, w_bytes = size_t(L->N) * L->C;
+        uint8_t* buf = nullptr;
+        int rc = stream_scratch(kScratchExpand, st, a_bytes + w_bytes, &buf);
+        if (rc != QLLM_OK) return rc;
+        QLLM_CUDA_TRY(cudaEventRecord(L->ev_fork, st));           // earlier users of the scratch are done
+        QLLM_CUDA_TRY(cudaStreamWaitEvent(L->side, L->ev_fork, 0));
+        rc = launch_expand_codes(L->w_codes, L->N, L->C, buf + a_bytes, L->side);
+        if (rc != QLLM_OK) return rc;
+        QLLM_CUDA_TRY(cudaEventRecord(L->ev_join, L->side));
+        L->w_ready = buf + a_bytes;
+        L->w_ready_M = M;
+    }
     return reassemble_entry(x, L->x_dtype, M, L->C, L->gamma, L->beta, L->eps, L->ptr, L->src, L->coef,
                             L->a_bits, L->map_image, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream);
 }
@@ -293,8 +331,15 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
 int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {
     if (!L || !out) return QLLM_ERR_NULL;
     if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
-    return qllm_qgemm(L->codes, L->a_scale, L->a_zero, L->w_codes, L->w_scale, L->w_zero, L->w_colsum,
-                      L->bias, out, M, L->N, L->C, L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum, stream);
+    const uint8_t* w_ready = nullptr;
+    if (L->w_ready && L->w_ready_M == M) {
+        QLLM_CUDA_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), L->ev_join, 0));
+        w_ready = L->w_ready;
+    }
+    L->w_ready = nullptr;
+    return gemm_entry(L->codes, L->a_scale, L->a_zero, L->w_codes, L->w_scale, L->w_zero, L->w_colsum, L->bias,
+                      out, M, L->N, L->C, L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum,
+                      static_cast<cudaStream_t>(stream), true, w_ready);
 }
 
 int qllm_layer_forward(qllm_layer_t* L, const void* x, int64_t M, void* out, void* stream) {
