@@ -115,7 +115,10 @@ int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C,
  *            calls needed, so pass a_rowsum on allocation-free paths).
  *  K must be even when either operand is 4-bit.  |I| must fit an int32.
  *  Dispatch: M <= 16 takes a weight-streaming kernel (weights read once); larger M takes the
- *  tensor-core kernel when the shape allows it, else a plain kernel.
+ *  tensor-core kernel when the shape allows it, else a plain kernel.  With a 4-bit operand and
+ *  M >= 512 the 4-bit codes are first widened to byte lanes, once per call, into a second
+ *  library-owned scratch buffer kept per (device, stream) and grown with cudaMalloc like the
+ *  row-sum scratch (N*K + M*K bytes at most); qllm_qgemm_noalloc never does this.
  */
 int qllm_qgemm(const uint8_t* codes, const float* a_scale, const float* a_zero,
                const uint8_t* w_codes, const float* w_scale, const float* w_zero,
