@@ -245,9 +245,13 @@ int qllm_layer_qgemm(qllm_layer_t* layer, int64_t M, void* out, void* stream);
  * path, copies out back and waits for the stream. */
 int qllm_layer_forward_host(qllm_layer_t* layer, const void* x_host, int64_t M, void* out_host,
                             void* stream);
-/* Borrowed DEVICE pointers of the layer's quantized-activation workspace of the last forward. */
+/* Borrowed DEVICE pointers of the layer's quantized-activation workspace of the last forward.
+ * *lane_bits (may be NULL) receives how the codes are stored: 4 = two per byte as qllm_reassemble_quant
+ * writes 4-bit codes, 8 = one per byte [M][C].  4-bit activations are stored one per byte when the
+ * call's GEMM runs on byte lanes (M >= 512 on the tensor-core path): the pre-GEMM kernel then writes
+ * the lanes the GEMM reads, which saves a widening pass; the code VALUES are the same. */
 int qllm_layer_workspace(qllm_layer_t* layer, uint8_t** codes, float** a_scale, float** a_zero,
-                         int32_t** a_rowsum);
+                         int32_t** a_rowsum, int* lane_bits);
 
 /* ==========================================================================
  * 6. Diagnostics

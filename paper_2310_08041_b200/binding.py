@@ -65,7 +65,8 @@ _lib.qllm_layer_forward.argtypes = [_vp, _vp, _i64, _vp, _vp]
 _lib.qllm_layer_forward_host.argtypes = [_vp, _vp, _i64, _vp, _vp]
 _lib.qllm_layer_reassemble_quant.argtypes = [_vp, _vp, _i64, _vp]
 _lib.qllm_layer_qgemm.argtypes = [_vp, _i64, _vp, _vp]
-_lib.qllm_layer_workspace.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp)]
+_lib.qllm_layer_workspace.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp),
+                                      ctypes.POINTER(ctypes.c_int)]
 _lib.qllm_status_string.argtypes = [_i]
 _lib.qllm_status_string.restype = ctypes.c_char_p
 _lib.qllm_launch_count.restype = _i64
@@ -290,6 +291,8 @@ class Layer:
         _check(_lib.qllm_layer_forward_host(self._h, hptr(x_host), M, hptr(out_host), _stream(stream)))
 
     def workspace_ptrs(self):
-        c, s, z, r = _vp(), _vp(), _vp(), _vp()
-        _check(_lib.qllm_layer_workspace(self._h, ctypes.byref(c), ctypes.byref(s), ctypes.byref(z), ctypes.byref(r)))
-        return c.value, s.value, z.value, r.value
+        """(codes, a_scale, a_zero, a_rowsum, lane_bits): device addresses and the code lane width (4 or 8)."""
+        c, s, z, r, lanes = _vp(), _vp(), _vp(), _vp(), ctypes.c_int(0)
+        _check(_lib.qllm_layer_workspace(self._h, ctypes.byref(c), ctypes.byref(s), ctypes.byref(z), ctypes.byref(r),
+                                         ctypes.byref(lanes)))
+        return c.value, s.value, z.value, r.value, lanes.value

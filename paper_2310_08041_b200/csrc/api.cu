@@ -160,6 +160,9 @@ struct qllm_layer {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     const uint8_t* w_ready = nullptr;            // expanded weights in flight / ready for the next GEMM call
     int64_t w_ready_M = -1;
+    // 4-bit activations of a call that will take the byte-lane GEMM are written one code per byte by the
+    // pre-GEMM kernel itself (no expansion pass): lane width of the codes now in the workspace
+    int lane_bits = 0;
     std::vector<void*> owned;
 };
 
@@ -187,7 +190,8 @@ extern "C" {
 static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
                             const float* ln_beta, float ln_eps, const int32_t* map_ptr,
                             const int32_t* map_src, const float* map_coef, int bits, const void* map_image,
-                            uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream) {
+                            uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream,
+                            bool byte_lanes = false) {
     if (!bits_ok(bits)) return QLLM_ERR_BITS;
     if (!dtype_ok(x_dtype)) return QLLM_ERR_DTYPE;
     if (M < 0 || C <= 0 || C > 49152 || (bits == 4 && (C & 1))) return QLLM_ERR_SHAPE;
@@ -197,7 +201,7 @@ static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const 
     if (!aligned16(x) || !aligned16(codes)) return QLLM_ERR_ALIGN;
     return launch_reassemble_quant(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, map_ptr, map_src,
                                    map_coef, bits, map_image, codes, a_scale, a_zero, a_rowsum,
-                                   static_cast<cudaStream_t>(stream));
+                                   static_cast<cudaStream_t>(stream), byte_lanes);
 }
 
 int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
@@ -276,7 +280,7 @@ int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const f
         if (rc == QLLM_OK) step(compile_reassemble_map(C, L->gamma, L->beta, L->ptr, L->src, L->coef, L->map_image, nullptr));
         if (rc == QLLM_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) rc = QLLM_ERR_CUDA;
     }
-    step(dev_alloc(L, &L->codes, size_t(max_M) * size_t(code_row_bytes(C, a_bits))));
+    step(dev_alloc(L, &L->codes, size_t(max_M) * size_t(C)));   // room for one code per byte
     step(dev_alloc(L, &L->a_scale, size_t(max_M)));
     step(dev_alloc(L, &L->a_zero, size_t(max_M)));
     step(dev_alloc(L, &L->a_rowsum, size_t(max_M)));
@@ -309,10 +313,13 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
     if (!L || !x) return QLLM_ERR_NULL;
     if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
     L->w_ready = nullptr;
-    if (L->side && expand_path(M, L->N, L->C, L->a_bits, L->w_bits)) {
+    const bool expand = expand_path(M, L->N, L->C, L->a_bits, L->w_bits);
+    const bool byte_lanes = expand && L->a_bits == 4 && reassemble_byte_lanes_supported(L->C);
+    L->lane_bits = (L->a_bits == 4 && !byte_lanes) ? 4 : 8;
+    if (L->side && expand) {
         // start expanding the weights for the coming GEMM on the side stream: it is independent of the tokens
         cudaStream_t st = static_cast<cudaStream_t>(stream);
-        const size_t a_bytes = L->a_bits == 4 ? size_t(M) * L->C : 0, w_bytes = size_t(L->N) * L->C;
+        const size_t a_bytes = L->lane_bits == 4 ? size_t(M) * L->C : 0, w_bytes = size_t(L->N) * L->C;
         uint8_t* buf = nullptr;
         int rc = stream_scratch(kScratchExpand, st, a_bytes + w_bytes, &buf);
         if (rc != QLLM_OK) return rc;
@@ -325,7 +332,8 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
         L->w_ready_M = M;
     }
     return reassemble_entry(x, L->x_dtype, M, L->C, L->gamma, L->beta, L->eps, L->ptr, L->src, L->coef,
-                            L->a_bits, L->map_image, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream);
+                            L->a_bits, L->map_image, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream,
+                            byte_lanes);
 }
 
 int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {
@@ -338,7 +346,7 @@ int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {
     }
     L->w_ready = nullptr;
     return gemm_entry(L->codes, L->a_scale, L->a_zero, L->w_codes, L->w_scale, L->w_zero, L->w_colsum, L->bias,
-                      out, M, L->N, L->C, L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum,
+                      out, M, L->N, L->C, L->lane_bits == 8 ? 8 : L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum,
                       static_cast<cudaStream_t>(stream), true, w_ready);
 }
 
@@ -363,8 +371,10 @@ int qllm_layer_forward_host(qllm_layer_t* L, const void* x_host, int64_t M, void
     return QLLM_OK;
 }
 
-int qllm_layer_workspace(qllm_layer_t* L, uint8_t** codes, float** a_scale, float** a_zero, int32_t** a_rowsum) {
+int qllm_layer_workspace(qllm_layer_t* L, uint8_t** codes, float** a_scale, float** a_zero, int32_t** a_rowsum,
+                         int* lane_bits) {
     if (!L) return QLLM_ERR_NULL;
+    if (lane_bits) *lane_bits = L->lane_bits;
     if (codes) *codes = L->codes;
     if (a_scale) *a_scale = L->a_scale;
     if (a_zero) *a_zero = L->a_zero;

@@ -63,12 +63,14 @@ int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out);
 // The specialised fused kernel consumes a compiled image of the reassembly map (0 bytes: the channel
 // count has no specialised kernel).  map_image = nullptr compiles one per call into stream scratch.
 size_t reassemble_map_image_bytes(int C);
+// true when the fused kernel for C channels can write 4-bit codes one per byte (byte_lanes below)
+bool reassemble_byte_lanes_supported(int C);
 int compile_reassemble_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
                            const float* coef, void* image, cudaStream_t st);
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                             const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
-                            float* a_zero, int32_t* a_rowsum, cudaStream_t st);
+                            float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes = false);
 int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                                     const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                                     const float* coef, int bits, uint8_t* codes, float* a_scale,
@@ -87,6 +89,10 @@ int launch_qgemm_plain(const uint8_t* a, const uint8_t* w, int64_t M, int N, int
 int launch_qgemm_decode(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
                         int w_bits, const EpilogueArgs& ep, cudaStream_t st);
 bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits);
+// CTA-pair (cta_group::2) variant for byte-lane codes on both operands and M > 128
+bool qgemm_tc2_supported(int64_t M, int N, int K, int a_bits, int w_bits);
+int launch_qgemm_tc2(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const EpilogueArgs& ep,
+                     cudaStream_t st);
 int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
                     int w_bits, const EpilogueArgs& ep, cudaStream_t st);
 bool qgemm_decode_supported(int64_t M, int N, int K, int a_bits, int w_bits);

@@ -244,6 +244,7 @@ int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K,
     const bool ap = a_bits == 4, wp = w_bits == 4;
     if (ap && wp) return launch<256, true, true>(a, w, M, N, K, ep, st);
     if (!ap && !wp) {
+        if (qgemm_tc2_supported(M, N, K, a_bits, w_bits)) return launch_qgemm_tc2(a, w, M, N, K, ep, st);
         // tile width that wastes the least of the last wave: cost ~ rounds x tile width
         const int64_t tm = (M + BM - 1) / BM;
         const int sms = sm_count();

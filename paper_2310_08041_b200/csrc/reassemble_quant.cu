@@ -432,12 +432,13 @@ int launch_main(const void* x, int64_t M, int C, const float* gamma, float eps, 
 
 template <int CPT, int NTT, typename XT>
 int launch_layout(const void* x, int64_t M, int C, const float* gamma, bool has_beta, float eps,
-                  const int32_t* ptr, const int32_t* src, const float* coef, int bits, const MapImage& im,
-                  uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
+                  const int32_t* ptr, const int32_t* src, const float* coef, int bits, bool packed,
+                  const MapImage& im, uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum,
+                  cudaStream_t st) {
 #define QLLM_MAIN(B, F) launch_main<CPT, NTT, XT, B, F>(x, M, C, gamma, eps, ptr, src, coef, bits, im, codes, a_scale, a_zero, a_rowsum, st)
     // run-time thread counts keep one variant per bit packing (the bias registers are always present)
-    if (NTT == 0 || has_beta) return bits == 4 ? QLLM_MAIN(true, true) : QLLM_MAIN(true, false);
-    return bits == 4 ? QLLM_MAIN(false, true) : QLLM_MAIN(false, false);
+    if (NTT == 0 || has_beta) return packed ? QLLM_MAIN(true, true) : QLLM_MAIN(true, false);
+    return packed ? QLLM_MAIN(false, true) : QLLM_MAIN(false, false);
 #undef QLLM_MAIN
 }
 
@@ -449,6 +450,8 @@ int layout_cpt(int C) {
 }
 
 }  // namespace
+
+bool reassemble_byte_lanes_supported(int C) { return layout_cpt(C) != 0; }
 
 size_t reassemble_map_image_bytes(int C) {
     const int cpt = layout_cpt(C);
@@ -470,8 +473,10 @@ int compile_reassemble_map(int C, const float* gamma, const float* beta, const i
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                             const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
-                            float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
+                            float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes) {
     const int cpt = layout_cpt(C);
+    if (!cpt && byte_lanes && bits == 4) return QLLM_ERR_UNSUPPORTED;
+    const bool packed = bits == 4 && !byte_lanes;
     if (!cpt)
         return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
                                                a_scale, a_zero, a_rowsum, st);
@@ -487,7 +492,7 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
     }
     const MapImage im = map_image_at(const_cast<void*>(map_image), cpt, nt);
     const bool bf = x_dtype == QLLM_BF16, hb = beta != nullptr;
-#define QLLM_RQ_ARGS x, M, C, gamma, hb, eps, ptr, src, coef, bits, im, codes, a_scale, a_zero, a_rowsum, st
+#define QLLM_RQ_ARGS x, M, C, gamma, hb, eps, ptr, src, coef, bits, packed, im, codes, a_scale, a_zero, a_rowsum, st
     // LLaMA hidden sizes get compile-time thread counts (immediate offsets, unrolled reductions)
     if (bf && C == 4096) return launch_layout<16, 256, __nv_bfloat16>(QLLM_RQ_ARGS);
     if (bf && C == 5120) return launch_layout<16, 320, __nv_bfloat16>(QLLM_RQ_ARGS);
