@@ -71,6 +71,41 @@ def test_odd_channel_count_byte_codes():
     parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref, 6)
 
 
+@pytest.mark.parametrize("kind", ["long_rows", "slot_overflow", "identity"])
+@pytest.mark.parametrize("with_beta", [False, True])
+def test_handmade_maps_on_the_specialised_kernel(kind, with_beta):
+    """Maps the builder would rarely produce, on a channel count the warp-per-token kernel serves:
+    rows with more entries than a slot record holds, more multi-entry rows than there are slots
+    (the launch then walks the CSR arrays), and the identity map."""
+    import gpu_util as G
+    rng = np.random.default_rng(11)
+    C = 512 if kind != "slot_overflow" else 4608
+    M = 21
+    x = (rng.standard_normal((M, C)) * (1 + 30 * (rng.random(C) < 0.01))).astype(np.float32)
+    if not with_beta:
+        x = synth.f32_to_bf16_bits(x)                    # bf16 rows without beta, fp32 rows with beta
+    g = (1 + 0.1 * rng.standard_normal(C)).astype(np.float32)
+    b = (0.05 * rng.standard_normal(C)).astype(np.float32) if with_beta else None
+    rows = []
+    for c in range(C):
+        if kind == "identity":
+            rows.append([(c, 1.0)])
+        elif kind == "long_rows":
+            n = 1 + (c % 9 == 0) * (1 + c % 7)           # rows of 1 .. 7 entries
+            srcs = [(c * 5 + 13 * e) % C for e in range(n)]
+            rows.append([(sj, 1.0 / n) for sj in srcs])
+        else:
+            rows.append([(c, 0.5), ((c * 7 + 3) % C, 0.5)])
+    ptr = np.zeros(C + 1, np.int32)
+    ptr[1:] = np.cumsum([len(r) for r in rows])
+    src = np.array([sj for r in rows for sj, _ in r], np.int32)
+    coef = np.array([cj for r in rows for _, cj in r], np.float32)
+    for bits in (4, 6):
+        got = G.run_reassemble_quant(x, g, b, 1e-5, ptr, src, coef, bits)
+        ref = oracle.reassemble_quant(x, g, b, 1e-5, ptr, src, coef, bits, want_pre=True)
+        parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref, bits)
+
+
 def test_degenerate_rows_and_empty_batch():
     import torch
     import gpu_util as G
