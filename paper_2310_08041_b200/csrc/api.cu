@@ -192,7 +192,7 @@ static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const 
                             const float* ln_beta, float ln_eps, const int32_t* map_ptr,
                             const int32_t* map_src, const float* map_coef, int bits, const void* map_image,
                             uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream,
-                            bool byte_lanes = false, int slots_known = -1) {
+                            bool byte_lanes = false, int slots_known = -1, bool share_sm = false) {
     if (!bits_ok(bits)) return QLLM_ERR_BITS;
     if (!dtype_ok(x_dtype)) return QLLM_ERR_DTYPE;
     if (M < 0 || C <= 0 || C > 49152 || (bits == 4 && (C & 1))) return QLLM_ERR_SHAPE;
@@ -202,7 +202,7 @@ static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const 
     if (!aligned16(x) || !aligned16(codes)) return QLLM_ERR_ALIGN;
     return launch_reassemble_quant(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, map_ptr, map_src,
                                    map_coef, bits, map_image, codes, a_scale, a_zero, a_rowsum,
-                                   static_cast<cudaStream_t>(stream), byte_lanes, slots_known);
+                                   static_cast<cudaStream_t>(stream), byte_lanes, slots_known, share_sm);
 }
 
 int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
@@ -334,7 +334,7 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
     }
     return reassemble_entry(x, L->x_dtype, M, L->C, L->gamma, L->beta, L->eps, L->ptr, L->src, L->coef,
                             L->a_bits, L->map_image, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream,
-                            byte_lanes, L->map_image ? L->map_slots : -1);
+                            byte_lanes, L->map_image ? L->map_slots : -1, L->w_ready != nullptr);
 }
 
 int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {

@@ -696,13 +696,26 @@ int launch_warp(const void* x, int64_t M, int C, float eps, int bits, const Warp
 
 template <int NPL, int G, bool HAS_BETA, bool PACKED, int MAXW>
 int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage& im, int slot_room, const RawMap& rm,
-                 uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
+                 uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool share_sm) {
     constexpr int C = NPL * 32 * G;
     auto kern = reassemble_quant_token<NPL, G, HAS_BETA, PACKED, MAXW>;
     const int row_words = C + slot_room;
     const int64_t fixed = int64_t(HAS_BETA ? 12 : 8) * C + (MAXW / G) * 8 * G * 4 + int64_t(slot_room) * 32;   // records, exchange, slot records
     int tok_fit = int((kSmemBudget - fixed) / (int64_t(row_words) * 4));
     if (tok_fit > MAXW / G) tok_fit = MAXW / G;
+    if (share_sm) {
+        // leave a fifth of the register file free: the layer expands its 4-bit weights for the coming GEMM
+        // on a second stream meanwhile, and that bandwidth-bound kernel needs room on every SM to keep
+        // enough loads in flight (this kernel is latency-bound and does not miss the token slot)
+        static int regs = 0;
+        if (regs == 0) {
+            cudaFuncAttributes fa;
+            QLLM_CUDA_TRY(cudaFuncGetAttributes(&fa, kern));
+            regs = fa.numRegs > 0 ? fa.numRegs : 128;
+        }
+        const int w_cap = int(0.8 * 65536 / (regs * 32));
+        if (tok_fit > w_cap / G && w_cap / G >= 1) tok_fit = w_cap / G;
+    }
     if (tok_fit < 1) return QLLM_ERR_UNSUPPORTED;
     const int sms = sm_count_rq();
     const int grid = int(M < sms ? M : sms);
@@ -737,8 +750,8 @@ int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage&
 template <int NPL, int G, int MAXW>
 int launch_token_variant(bool has_beta, bool packed, const void* x, int64_t M, float eps, int bits,
                          const WarpImage& im, int slot_room, const RawMap& rm, uint8_t* codes, float* a_scale,
-                         float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
-#define QLLM_RQT(B, P) launch_token<NPL, G, B, P, MAXW>(x, M, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st)
+                         float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool share_sm) {
+#define QLLM_RQT(B, P) launch_token<NPL, G, B, P, MAXW>(x, M, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm)
     if (has_beta) return packed ? QLLM_RQT(true, true) : QLLM_RQT(true, false);
     return packed ? QLLM_RQT(false, true) : QLLM_RQT(false, false);
 #undef QLLM_RQT
@@ -777,7 +790,8 @@ int reassemble_map_slots(int C, const void* image, cudaStream_t st, int* slots) 
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                             const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
-                            float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes, int slots_known) {
+                            float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes, int slots_known,
+                            bool share_sm) {
     if (!warp_kernel_serves(C)) {
         if (byte_lanes && bits == 4) return QLLM_ERR_UNSUPPORTED;
         return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
@@ -800,7 +814,7 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
     const bool packed = bits == 4 && !byte_lanes, has_beta = beta != nullptr;
     if (x_dtype == QLLM_BF16) {
         // LLaMA hidden sizes: shape fixed at compile time
-#define QLLM_TOKEN_ARGS has_beta, packed, x, M, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st
+#define QLLM_TOKEN_ARGS has_beta, packed, x, M, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm
         if (M <= sm_count_rq()) {                          // one token per CTA: spread it over more warps
             if (C == 4096) return launch_token_variant<16, 8, 8>(QLLM_TOKEN_ARGS);
             if (C == 5120) return launch_token_variant<40, 4, 4>(QLLM_TOKEN_ARGS);
