@@ -246,8 +246,8 @@ def run_gpu(args):
                         "traffic": None}
         else:
             expand = (cfg.a_bits == 4 or cfg.w_bits == 4) and M >= 512
-            roofline = {"kernel": "qllm_qgemm call: " + ("2 expand_codes launches + " if expand else "") +
-                                  "qgemm_tc_kernel (tcgen05 kind::i8) + dequant epilogue",
+            roofline = {"kernel": "qllm_layer_qgemm: " + ("join of the side-stream weight expansion + " if expand and cfg.w_bits == 4 else "") +
+                                  "qgemm_tc2_kernel (tcgen05 kind::i8, cta_group::2, byte lanes) + dequant epilogue",
                         "bound": "tensor", "achieved": tops, "peak": int8_peak, "unit": "TOP/s", "frac": tops / int8_peak,
                         "peak_source": f"2 x {peaks['source']} bf16 burst ({peaks['bf16_burst']} TFLOP/s); nominal int8:bf16 = 2",
                         "frac_of_nominal_4500": tops / 4500.0, "ms": ms_gemm, "traffic": None}
