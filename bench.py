@@ -24,6 +24,9 @@ if ROOT not in sys.path:
 
 METRIC = "W4A4 reassembled-linear tokens/s; TOPS & GB/s as % of B200 roofline"
 UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the GEMM kernel, from the ncu captures summarised
+# under profiles/ (keyed by workload and tokens per GPU; absent = not captured for the current kernel)
+NCU_TRAFFIC = {("c2", 2048): 72.0e6, ("c3", 16): 45.4e6}
 
 
 def _peaks():
@@ -243,14 +246,14 @@ def run_gpu(args):
             roofline = {"kernel": "qllm_qgemm call: qgemm_decode_kernel (weight streaming)", "bound": "hbm",
                         "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                         "peak_source": f"{peaks['source']} STREAM-style copy", "ms": ms_gemm, "bytes": gemm_bytes,
-                        "traffic": None}
+                        "traffic": NCU_TRAFFIC.get((cfg.name, M))}
         else:
             expand = (cfg.a_bits == 4 or cfg.w_bits == 4) and M >= 512
             roofline = {"kernel": "qllm_layer_qgemm: " + ("join of the side-stream weight expansion + " if expand and cfg.w_bits == 4 else "") +
                                   "qgemm_tc2_kernel (tcgen05 kind::i8, cta_group::2, byte lanes) + dequant epilogue",
                         "bound": "tensor", "achieved": tops, "peak": int8_peak, "unit": "TOP/s", "frac": tops / int8_peak,
                         "peak_source": f"2 x {peaks['source']} bf16 burst ({peaks['bf16_burst']} TFLOP/s); nominal int8:bf16 = 2",
-                        "frac_of_nominal_4500": tops / 4500.0, "ms": ms_gemm, "traffic": None}
+                        "frac_of_nominal_4500": tops / 4500.0, "ms": ms_gemm, "traffic": NCU_TRAFFIC.get((cfg.name, M))}
         line = {
             "metric": METRIC, "value": world * M / (ms_step_w * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step_w, "higher_is_better": True,

@@ -105,43 +105,52 @@ qgemm_decode_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ w
     fill_tokens<WP>(As, stride, a, M, K, a_bits, M16 ? 16 : 8);
     __syncthreads();
 
+    // One step of the stream: UN x 16 bytes of this thread's weight column against the matching token
+    // fragments.  Loads past the end of the row return zeros, so a step needs no bounds test: zero weights
+    // add nothing (the token fragments then come from the slack behind the last row).  Two accumulator sets
+    // halve the chain of dependent MMAs.
+    auto step = [&](const uint4 (&buf)[UN], int it0, int (&c0)[4], int (&c1)[4]) {
+#pragma unroll
+        for (int u = 0; u < UN; ++u) {
+            const int it = it0 + u;
+            const uint4 wv = buf[u];
+            if (WP) {
+                // 32 codes of this thread's column: words s = 0..3, each -> (even, odd) registers
+                const int aoff = (16 * it + 4 * tig) * 8;
+                const uint4 A0 = *reinterpret_cast<const uint4*>(a_lo + aoff);
+                const uint4 A1 = *reinterpret_cast<const uint4*>(a_lo + aoff + 16);
+                uint4 B0 = make_uint4(0, 0, 0, 0), B1 = B0;
+                if (M16) {
+                    B0 = *reinterpret_cast<const uint4*>(a_hi + aoff);
+                    B1 = *reinterpret_cast<const uint4*>(a_hi + aoff + 16);
+                }
+                mma_u8(c0, A0.x, B0.x, A0.y, B0.y, wv.x & 0x0F0F0F0Fu, (wv.x >> 4) & 0x0F0F0F0Fu);
+                mma_u8(c1, A0.z, B0.z, A0.w, B0.w, wv.y & 0x0F0F0F0Fu, (wv.y >> 4) & 0x0F0F0F0Fu);
+                mma_u8(c0, A1.x, B1.x, A1.y, B1.y, wv.z & 0x0F0F0F0Fu, (wv.z >> 4) & 0x0F0F0F0Fu);
+                mma_u8(c1, A1.z, B1.z, A1.w, B1.w, wv.w & 0x0F0F0F0Fu, (wv.w >> 4) & 0x0F0F0F0Fu);
+            } else {
+                // 16 byte codes of this thread's column: two k32 steps
+                const int aoff = (4 * it + tig) * 16;
+                const uint4 A0 = *reinterpret_cast<const uint4*>(a_lo + aoff);
+                uint4 B0 = make_uint4(0, 0, 0, 0);
+                if (M16) B0 = *reinterpret_cast<const uint4*>(a_hi + aoff);
+                mma_u8(c0, A0.x, B0.x, A0.y, B0.y, wv.x, wv.y);
+                mma_u8(c1, A0.z, B0.z, A0.w, B0.w, wv.z, wv.w);
+            }
+        }
+    };
+
     for (; task < tasks; task += gridDim.x * nwarps) {
         const int n_base = task * 8;
-        int c[4] = {0, 0, 0, 0};
-        for (int it0 = 0; it0 < iters; it0 += UN) {
+        int c[4] = {0, 0, 0, 0}, c2[4] = {0, 0, 0, 0};
+        for (int it0 = 0; it0 < iters; it0 += 2 * UN) {
             load_block(nxt, wp, it0 + UN);        // zeros past the end of the row
-#pragma unroll
-            for (int u = 0; u < UN; ++u) {
-                const int it = it0 + u;
-                if (it >= iters) break;
-                const uint4 wv = cur[u];
-                if (WP) {
-                    // 32 codes of this thread's column: words s = 0..3, each -> (even, odd) registers
-                    const int aoff = (16 * it + 4 * tig) * 8;
-                    const uint4 A0 = *reinterpret_cast<const uint4*>(a_lo + aoff);
-                    const uint4 A1 = *reinterpret_cast<const uint4*>(a_lo + aoff + 16);
-                    uint4 B0 = make_uint4(0, 0, 0, 0), B1 = B0;
-                    if (M16) {
-                        B0 = *reinterpret_cast<const uint4*>(a_hi + aoff);
-                        B1 = *reinterpret_cast<const uint4*>(a_hi + aoff + 16);
-                    }
-                    mma_u8(c, A0.x, B0.x, A0.y, B0.y, wv.x & 0x0F0F0F0Fu, (wv.x >> 4) & 0x0F0F0F0Fu);
-                    mma_u8(c, A0.z, B0.z, A0.w, B0.w, wv.y & 0x0F0F0F0Fu, (wv.y >> 4) & 0x0F0F0F0Fu);
-                    mma_u8(c, A1.x, B1.x, A1.y, B1.y, wv.z & 0x0F0F0F0Fu, (wv.z >> 4) & 0x0F0F0F0Fu);
-                    mma_u8(c, A1.z, B1.z, A1.w, B1.w, wv.w & 0x0F0F0F0Fu, (wv.w >> 4) & 0x0F0F0F0Fu);
-                } else {
-                    // 16 byte codes of this thread's column: two k32 steps
-                    const int aoff = (4 * it + tig) * 16;
-                    const uint4 A0 = *reinterpret_cast<const uint4*>(a_lo + aoff);
-                    uint4 B0 = make_uint4(0, 0, 0, 0);
-                    if (M16) B0 = *reinterpret_cast<const uint4*>(a_hi + aoff);
-                    mma_u8(c, A0.x, B0.x, A0.y, B0.y, wv.x, wv.y);
-                    mma_u8(c, A0.z, B0.z, A0.w, B0.w, wv.z, wv.w);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < UN; ++u) cur[u] = nxt[u];
+            step(cur, it0, c, c2);
+            load_block(cur, wp, it0 + 2 * UN);
+            step(nxt, it0 + UN, c, c2);
         }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) c[q] += c2[q];
         // next task's first block (if any) while this task's results are written
         const int next_task = task + gridDim.x * nwarps;
         if (next_task < tasks) { wp = row_ptr(next_task); load_block(cur, wp, 0); }
@@ -199,7 +208,8 @@ template <bool WP, bool M16>
 int launch(const uint8_t* a, const uint8_t* w, int M, int N, int K, int a_bits, const EpilogueArgs& ep,
            cudaStream_t st) {
     auto kern = qgemm_decode_kernel<WP, M16>;
-    const size_t smem = size_t(M16 ? 16 : 8) * size_t(K + (WP ? 16 : 64));
+    // + slack: the last steps of a row may read token fragments up to 8 iterations (1 KB) past the last row
+    const size_t smem = size_t(M16 ? 16 : 8) * size_t(K + (WP ? 16 : 64)) + 1024;
     QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     const int tasks = (N + 7) / 8;
     const int sms = sm_count();
@@ -214,7 +224,7 @@ int launch(const uint8_t* a, const uint8_t* w, int M, int N, int K, int a_bits, 
 bool qgemm_decode_supported(int64_t M, int N, int K, int a_bits, int w_bits) {
     (void)a_bits; (void)w_bits;
     if (M < 1 || M > 16 || N < 1 || K % 128 != 0) return false;
-    return size_t(16) * size_t(K + 64) <= 200 * 1024;
+    return size_t(16) * size_t(K + 64) + 1024 <= 200 * 1024;
 }
 
 int launch_qgemm_decode(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,

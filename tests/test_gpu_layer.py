@@ -65,7 +65,7 @@ def test_layer_forward_matches_oracle(name, kw, out_dtype):
     layer.destroy()
 
 
-@pytest.mark.parametrize("name", ["c2", "c4", "c5"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
 def test_layer_full_size_two_halves_sampled(name):
     """The launch configuration the benchmark times: layer object, full-size workload, the two half-step
     calls.  Activation codes are compared in full under the flip rule (whatever lane width the layer
