@@ -5,7 +5,7 @@ A step = one pass of the whole path over one batch of synthetic tokens: the fuse
 LayerNorm + reassembly + quantization kernel, then the integer GEMM with its dequantizing
 epilogue.  Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c4|c5] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5|c2_w4a8] [--impl reference]
 """
 from __future__ import annotations
 
@@ -290,7 +290,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c2_w4a8"])
     ap.add_argument("--ref-rows", type=int, default=0, help="token rows of the oracle sample (0 = auto)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -52,6 +52,9 @@ CONFIGS = {
                       n_outlier=25, outlier_lo=20.0, outlier_hi=100.0),
     "c5": LayerConfig("c5", M=4096, K=8192, N=10240, a_bits=4, w_bits=4, x_dtype="bf16", seed=5,
                       n_outlier=40, outlier_lo=20.0, outlier_hi=100.0, n_massive=2, w_std=0.015),
+    # the W4A8 setting of the paper's tables on the c2 shape: 8-bit activations, 4-bit weights
+    "c2_w4a8": LayerConfig("c2_w4a8", M=2048, K=4096, N=12288, a_bits=8, w_bits=4, x_dtype="bf16", seed=2,
+                           n_outlier=20, outlier_lo=20.0, outlier_hi=100.0),
 }
 
 

@@ -65,7 +65,7 @@ def test_layer_forward_matches_oracle(name, kw, out_dtype):
     layer.destroy()
 
 
-@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5", "c2_w4a8"])
 def test_layer_full_size_two_halves_sampled(name):
     """The launch configuration the benchmark times: layer object, full-size workload, the two half-step
     calls.  Activation codes are compared in full under the flip rule (whatever lane width the layer
@@ -106,7 +106,14 @@ def test_layer_full_size_two_halves_sampled(name):
     zero = from_dev(pz, (M,), "<f4")
     rowsum = from_dev(pr, (M,), "<i4")
     ref_q = oracle.reassemble_quant(x, L["gamma"], L["beta"], cfg.ln_eps, L["ptr"], L["src"], L["coef"], cfg.a_bits, want_pre=True)
-    parity.check_activation_codes(codes, scale, zero, rowsum, ref_q, cfg.a_bits)
+    # 8-bit codes: the pre-round values are 17x larger than 4-bit ones, so the fp32 error scales with them;
+    # the band is widened in proportion (255/15) for this bit-width only
+    old_band = parity.FLIP_BAND
+    parity.FLIP_BAND = old_band * (17 if cfg.a_bits == 8 else 1)
+    try:
+        parity.check_activation_codes(codes, scale, zero, rowsum, ref_q, cfg.a_bits)
+    finally:
+        parity.FLIP_BAND = old_band
     rng = np.random.default_rng(cfg.seed + 100)
     ms = np.concatenate([rng.integers(0, M, 600), [0, 0, M - 1, M - 1]]).astype(np.int64)
     ns = np.concatenate([rng.integers(0, N, 600), [0, N - 1, 0, N - 1]]).astype(np.int32)
