@@ -28,6 +28,18 @@ struct StreamScratch { cudaStream_t st; uint8_t* ptr; size_t cap; };
 std::vector<StreamScratch> g_stream_scratch[kScratchKinds][64];
 }  // namespace
 
+int device_sm_count() {
+    static std::atomic<int> cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+
 int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out) {
     int dev = 0;
     QLLM_CUDA_TRY(cudaGetDevice(&dev));

@@ -39,6 +39,9 @@ inline bool dtype_ok(int d) { return d == QLLM_F32 || d == QLLM_BF16; }
 // Bytes of one row of K codes at the given bit-width (4-bit codes are packed two per byte).
 inline int64_t code_row_bytes(int K, int bits) { return bits == 4 ? K / 2 : K; }
 
+// Number of SMs of the current device (cached per device; 148 if the query fails).
+int device_sm_count();
+
 // Device-side status word (one per loaded library image and device).
 int* device_status_word();          // device address, or nullptr on failure (error recorded)
 

@@ -180,17 +180,6 @@ qgemm_decode_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ w
     }
 }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            n = 148;
-    }
-    return n;
-}
-
 // Warps per CTA (one CTA per SM) that waste the fewest warp-slots in the last wave.
 int pick_warps(int tasks, int sms) {
     int best = kMaxWarps;
@@ -212,7 +201,7 @@ int launch(const uint8_t* a, const uint8_t* w, int M, int N, int K, int a_bits, 
     const size_t smem = size_t(M16 ? 16 : 8) * size_t(K + (WP ? 16 : 64)) + 1024;
     QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
     const int tasks = (N + 7) / 8;
-    const int sms = sm_count();
+    const int sms = device_sm_count();
     const int grid = std::min(sms, tasks);
     const int wpc = tasks <= sms * 8 ? 8 : pick_warps(tasks, sms);
     kern<<<grid, 32 * wpc, smem, st>>>(a, w, M, N, K, a_bits, ep, tasks);

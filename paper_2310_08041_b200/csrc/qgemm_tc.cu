@@ -227,7 +227,7 @@ int launch(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const Ep
     auto kern = qgemm_tc_kernel<BN, AP, WP>;
     QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM));
     const int64_t tiles = ((M + BM - 1) / BM) * int64_t((N + BN - 1) / BN);
-    const int grid = int(std::min<int64_t>(tiles, sm_count()));
+    const int grid = int(std::min<int64_t>(tiles, device_sm_count()));
     kern<<<grid, T::THREADS, T::SMEM, st>>>(tmA, tmW, M, N, K, ep, status);
     return after_launch();
 }
@@ -247,7 +247,7 @@ int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K,
         if (qgemm_tc2_supported(M, N, K, a_bits, w_bits)) return launch_qgemm_tc2(a, w, M, N, K, ep, st);
         // tile width that wastes the least of the last wave: cost ~ rounds x tile width
         const int64_t tm = (M + BM - 1) / BM;
-        const int sms = sm_count();
+        const int sms = device_sm_count();
         auto cost = [&](int bn) {
             const int64_t tiles = tm * ((N + bn - 1) / bn);
             return ((tiles + sms - 1) / sms) * int64_t(bn + 16);   // + per-tile fill/drain overhead

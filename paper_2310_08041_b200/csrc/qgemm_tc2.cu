@@ -240,7 +240,7 @@ int launch_pair(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, con
     auto kern = qgemm_tc2_kernel<BN>;
     QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM));
     const int64_t tiles = ((M + 2 * BM - 1) / (2 * BM)) * int64_t((N + BN - 1) / BN);
-    const int pairs = int(std::min<int64_t>(tiles, sm_count() / 2));
+    const int pairs = int(std::min<int64_t>(tiles, device_sm_count() / 2));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(unsigned(2 * pairs));
     cfg.blockDim = dim3(T::THREADS);
@@ -260,7 +260,7 @@ int launch_pair(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, con
 }  // namespace
 
 bool qgemm_tc2_supported(int64_t M, int N, int K, int a_bits, int w_bits) {
-    return a_bits != 4 && w_bits != 4 && M > BM && qgemm_tc_supported(M, N, K, a_bits, w_bits) && sm_count() >= 2;
+    return a_bits != 4 && w_bits != 4 && M > BM && qgemm_tc_supported(M, N, K, a_bits, w_bits) && device_sm_count() >= 2;
 }
 
 int launch_qgemm_tc2(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const EpilogueArgs& ep,
@@ -271,7 +271,7 @@ int launch_qgemm_tc2(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K
     // the constant stands for the per-tile fill/drain.  Measured per-MMA times (62 / 68 / 81 ns at
     // BN = 128 / 192 / 256) follow the same proportion.
     const int64_t tm = (M + 2 * BM - 1) / (2 * BM);
-    const int pairs = sm_count() / 2;
+    const int pairs = device_sm_count() / 2;
     auto cost = [&](int bn) {
         const int64_t tiles = tm * ((N + bn - 1) / bn);
         return ((tiles + pairs - 1) / pairs) * int64_t(256 + bn + 12);

@@ -656,17 +656,6 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
     }
 }
 
-int sm_count_rq() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            n = 148;
-    }
-    return n;
-}
-
 // warps per CTA that fit with the given slot room (0: does not fit)
 int warps_that_fit(int C, bool has_beta, int slot_room) {
     const int64_t rec = int64_t(has_beta ? 10 : 6) * C;
@@ -681,7 +670,7 @@ int launch_warp(const void* x, int64_t M, int C, float eps, int bits, const Warp
                 cudaStream_t st) {
     auto kern = reassemble_quant_warp<XT, HAS_BETA, PACKED>;
     const int wfit = warps_that_fit(C, HAS_BETA, slot_room);
-    const int sms = sm_count_rq();
+    const int sms = device_sm_count();
     const int grid = int(M < sms ? M : sms);
     const int64_t per_cta = (M + grid - 1) / grid;        // tokens a CTA gets
     const int W = int(per_cta < wfit ? per_cta : wfit);
@@ -717,7 +706,7 @@ int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage&
         if (tok_fit > w_cap / G && w_cap / G >= 1) tok_fit = w_cap / G;
     }
     if (tok_fit < 1) return QLLM_ERR_UNSUPPORTED;
-    const int sms = sm_count_rq();
+    const int sms = device_sm_count();
     const int grid = int(M < sms ? M : sms);
     const int64_t per_cta = (M + grid - 1) / grid;
     const int tok = int(per_cta < tok_fit ? per_cta : tok_fit);
@@ -815,7 +804,7 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
     if (x_dtype == QLLM_BF16) {
         // LLaMA hidden sizes: shape fixed at compile time
 #define QLLM_TOKEN_ARGS has_beta, packed, x, M, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm
-        if (M <= sm_count_rq()) {                          // one token per CTA: spread it over more warps
+        if (M <= device_sm_count()) {                          // one token per CTA: spread it over more warps
             if (C == 4096) return launch_token_variant<16, 8, 8>(QLLM_TOKEN_ARGS);
             if (C == 5120) return launch_token_variant<40, 4, 4>(QLLM_TOKEN_ARGS);
             if (C == 8192) return launch_token_variant<16, 16, 16>(QLLM_TOKEN_ARGS);

@@ -132,16 +132,6 @@ calib_absmax_kernel(const XT* __restrict__ x, int64_t M, int C, const float* __r
         atomicMax(reinterpret_cast<int*>(absmax + k), __float_as_int(amax[k]));
 }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n = 148;
-    }
-    return n;
-}
-
 }  // namespace
 
 int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
@@ -150,7 +140,7 @@ int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C
                                     float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
     const size_t smem = size_t(C) * sizeof(float);
     if (smem > 200 * 1024) return QLLM_ERR_UNSUPPORTED;
-    const int grid = int(std::min<int64_t>(M, int64_t(sm_count()) * 4));
+    const int grid = int(std::min<int64_t>(M, int64_t(device_sm_count()) * 4));
     if (x_dtype == QLLM_F32) {
         auto k = reassemble_quant_generic<float>;
         if (smem > 48 * 1024) QLLM_CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
@@ -169,7 +159,7 @@ int launch_calib_absmax(const void* x, int x_dtype, int64_t M, int C, const floa
                         const float* beta, float eps, float* absmax, cudaStream_t st) {
     const size_t smem = 2 * size_t(C) * sizeof(float);
     if (smem > 200 * 1024) return QLLM_ERR_UNSUPPORTED;
-    const int grid = int(std::min<int64_t>(M, int64_t(sm_count())));
+    const int grid = int(std::min<int64_t>(M, int64_t(device_sm_count())));
     if (x_dtype == QLLM_F32) {
         auto k = calib_absmax_kernel<float>;
         if (smem > 48 * 1024) QLLM_CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
