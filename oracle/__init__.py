@@ -237,3 +237,40 @@ def reassemble_quant(x, gamma, beta, eps, ptr, src, coef, bits, want_pre=False):
     q = quant_rows(xr, bits, want_pre=want_pre)
     q["xr"] = xr
     return q
+
+
+# ---------------------------------------------------------------------------
+# Adaptive threshold search (Algorithm 1), a composition of the steps above.
+# Reading: the reassembly error of Eq. 6 is taken on the layer's own output (the
+# calibration tokens through the full-precision layer against the same tokens
+# through the reassembled, quantized layer), not on an attention block's output.
+# ---------------------------------------------------------------------------
+def theta_grid(absmax, P):
+    """Algorithm 1: theta_p = min(m) + p / P * (max(m) - min(m)), p = 1..P (float32 values)."""
+    m = _c(absmax, np.float32).astype(np.float64)
+    lo, hi = float(m.min()), float(m.max())
+    return np.array([np.float32(lo + (p / P) * (hi - lo)) for p in range(1, P + 1)], np.float32)
+
+
+def reassembly_loss(xcal, gamma, beta, eps, W, absmax, theta, a_bits, w_bits):
+    """|| Y - Y~ ||_F^2 with Y = LN(x) W^T and Y~ = quant(X^) quant(W^) for the map built at theta
+    (Eq. 6 on the layer's output); inf when the channel count cannot be restored."""
+    y = layernorm(xcal, gamma, beta, eps)
+    Y = dense_linear(y, _c(W, np.float32).astype(np.float64))
+    try:
+        ptr, src, coef, _ = build_map(absmax, theta)
+    except Infeasible:
+        return float("inf")
+    w = prepare_weights(W, ptr, src, w_bits)
+    q = reassemble_quant(xcal, gamma, beta, eps, ptr, src, coef, a_bits)
+    acc = int_matmul(q["codes"], w["codes"])
+    Yq = epilogue(acc, W.shape[1], q["scale"], q["zero"], q["sum"], w["scale"], w["zero"], w["colsum"])
+    return float(((Y - Yq) ** 2).sum())
+
+
+def search_theta(xcal, gamma, beta, eps, W, absmax, a_bits, w_bits, P):
+    """Algorithm 1: returns (theta*, losses[P]); theta* is the first grid point with the smallest loss."""
+    grid = theta_grid(absmax, P)
+    losses = np.array([reassembly_loss(xcal, gamma, beta, eps, W, absmax, float(t), a_bits, w_bits) for t in grid])
+    best = int(np.argmin(losses))          # first occurrence: Algorithm 1 updates only on a strictly smaller loss
+    return float(grid[best]), losses

@@ -377,3 +377,59 @@ def test_theta_helpers():
         assert int((T - 1).sum()) == extra == oracle.extra_channels(a, th)
     # T rule of Sec. 4.1.1: below theta unchanged, above split by ceil
     assert oracle.extra_channels(np.array([1.0, 2.0, 2.0001, 7.9, 0.0], np.float32), 2.0) == 0 + 0 + 1 + 3 + 0
+
+
+# ---------------------------------------------------------------------------
+# Adaptive threshold search (Algorithm 1)
+# ---------------------------------------------------------------------------
+def _search_case(seed=7, T=24, C=64, N=40):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((T, C)).astype(np.float32)
+    x[:, [3, 17]] *= 30.0
+    gamma = (1 + 0.1 * rng.standard_normal(C)).astype(np.float32)
+    W = (0.05 * rng.standard_normal((N, C))).astype(np.float32)
+    absmax = oracle.channel_absmax(oracle.layernorm(x, gamma, None, 1e-5))
+    return x, gamma, W, absmax
+
+
+def test_theta_grid_closed_form():
+    """Algorithm 1: P evenly spaced thresholds ending at max(m); the first lies one step above min(m)."""
+    m = np.array([0.5, 4.0, 1.25, 2.0], np.float32)
+    g = oracle.theta_grid(m, 7)
+    assert g.shape == (7,) and g[-1] == np.float32(4.0)
+    np.testing.assert_allclose(np.diff(g.astype(np.float64)), 0.5, rtol=1e-6)
+    assert g[0] == np.float32(1.0)
+
+
+def test_reassembly_loss_without_outlier_channels_is_plain_quantization_error():
+    """At theta = max(m) every T_i = 1, the map is the identity, and the loss reduces to the error of
+    quantizing both operands: recomputed here from the dequantized operands with numpy."""
+    x, gamma, W, absmax = _search_case()
+    theta = float(absmax.max())
+    ptr, src, coef, st = oracle.build_map(absmax, theta)
+    assert st["E"] == 0 and np.array_equal(src, np.arange(len(absmax)))
+    y = oracle.layernorm(x, gamma, None, 1e-5)
+    qa = oracle.quant_rows(y, 4)
+    qw = oracle.quant_rows(W.astype(np.float64), 4)
+    A = qa["scale"].astype(np.float64)[:, None] * (qa["codes"].astype(np.float64) - qa["zero"].astype(np.float64)[:, None])
+    Wd = qw["scale"].astype(np.float64)[:, None] * (qw["codes"].astype(np.float64) - qw["zero"].astype(np.float64)[:, None])
+    want = float(((y @ W.astype(np.float64).T - A @ Wd.T) ** 2).sum())
+    got = oracle.reassembly_loss(x, gamma, None, 1e-5, W, absmax, theta, 4, 4)
+    assert abs(got - want) <= 1e-9 * want
+
+
+def test_search_theta_is_the_first_minimum_of_the_grid_losses():
+    x, gamma, W, absmax = _search_case()
+    P = 9
+    theta, losses = oracle.search_theta(x, gamma, None, 1e-5, W, absmax, 4, 4, P)
+    grid = oracle.theta_grid(absmax, P)
+    assert losses.shape == (P,)
+    finite = np.isfinite(losses)
+    assert finite[-1]                                   # theta = max(m) never needs assembly
+    best = min(range(P), key=lambda p: (losses[p], p))  # brute force with the tie rule of Algorithm 1
+    assert theta == float(grid[best])
+    # every finite loss is reproduced by evaluating its grid point on its own
+    for p in np.nonzero(finite)[0][:3]:
+        assert losses[p] == oracle.reassembly_loss(x, gamma, None, 1e-5, W, absmax, float(grid[p]), 4, 4)
+    # splitting the outlier channels helps on this input: some interior threshold beats "no reassembly"
+    assert losses[best] < losses[-1]
