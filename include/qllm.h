@@ -218,6 +218,22 @@ float qllm_theta_percentile(const float* absmax, int C, double pct);
  * thresholds on which E(theta) = extra.  Returns 0 when that interval is empty. */
 float qllm_theta_for_extra(const float* absmax, int C, int extra);
 
+/* Adaptive threshold search (Algorithm 1; host-orchestrated, offline, waits for the device).
+ * For p = 1..P the threshold theta_p = min(m) + p/P (max(m) - min(m)) over the calibration maxima m is tried:
+ * the reassembly is built (qllm_build_reassembly, no low-rank term: the search precedes error correction),
+ * the calibration tokens run through the reassembled, quantized layer (sections 1 + 2, fp32 output), and the
+ * reassembly error  L = || LayerNorm(x) W^T - quant(X^) quant(W^) ||_F^2  (Eq. 6, read on the layer's own
+ * output) is summed in fp64 against an fp32 reference product computed once.  *theta_out is the first
+ * threshold with the smallest error; losses_out[p-1] (host double[P], may be NULL) receives every error,
+ * +inf for a threshold whose map cannot restore the channel count.
+ *  calib_x   device [T][C] (x_dtype), 16-byte aligned, T <= 2^24
+ *  ln_gamma, ln_beta, calib_absmax, W   HOST (as for qllm_layer_create / qllm_build_reassembly)
+ * Allocates device memory for W, the reference and one layer object per candidate and frees it before
+ * returning. */
+int qllm_search_theta(const void* calib_x, int x_dtype, int64_t T, int C, const float* ln_gamma,
+                      const float* ln_beta, float ln_eps, const float* calib_absmax, const float* W, int N,
+                      int a_bits, int w_bits, int P, float* theta_out, double* losses_out, void* stream);
+
 /* ==========================================================================
  * 5. Layer object: device-resident map, weights and workspace
  * ==========================================================================

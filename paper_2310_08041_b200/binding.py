@@ -27,7 +27,7 @@ EXPORTS = [
     "qllm_reassemble_quant", "qllm_qgemm", "qllm_qgemm_noalloc", "qllm_qgemm_acc", "qllm_calib_absmax",
     "qllm_build_reassembly", "qllm_free_reassembly", "qllm_reassembly_map",
     "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map",
-    "qllm_theta_percentile", "qllm_theta_for_extra",
+    "qllm_theta_percentile", "qllm_theta_for_extra", "qllm_search_theta",
     "qllm_layer_create", "qllm_layer_destroy", "qllm_layer_forward", "qllm_layer_forward_host",
     "qllm_layer_reassemble_quant", "qllm_layer_qgemm",
     "qllm_layer_workspace",
@@ -56,6 +56,7 @@ _lib.qllm_reassembly_stats.argtypes = [_vp, ctypes.POINTER(_i64)]
 _lib.qllm_validate_map.argtypes = [_vp, _vp, _i, _i64]
 _lib.qllm_theta_percentile.argtypes = [_vp, _i, _d]
 _lib.qllm_theta_percentile.restype = _f
+_lib.qllm_search_theta.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]
 _lib.qllm_theta_for_extra.argtypes = [_vp, _i, _i]
 _lib.qllm_theta_for_extra.restype = _f
 _lib.qllm_layer_create.argtypes = [_vp, _vp, _vp, _f, _vp, _i, _i, _i, _i64, ctypes.POINTER(_vp)]
@@ -177,6 +178,23 @@ def qllm_theta_percentile(absmax, pct):
 def qllm_theta_for_extra(absmax, extra):
     a = np.ascontiguousarray(absmax, np.float32)
     return float(_lib.qllm_theta_for_extra(_hp(a), a.shape[0], extra))
+
+
+def qllm_search_theta(calib_x, ln_gamma, ln_beta, absmax, W, a_bits, w_bits, P, ln_eps=1e-5, stream=None):
+    """calib_x: device tensor [T][C]; ln_gamma, ln_beta (or None), absmax [C], W [N][C]: numpy (host).
+    Returns (theta, losses float64[P])."""
+    T, C = calib_x.shape
+    g = np.ascontiguousarray(ln_gamma, np.float32)
+    b = None if ln_beta is None else np.ascontiguousarray(ln_beta, np.float32)
+    a = np.ascontiguousarray(absmax, np.float32)
+    w = np.ascontiguousarray(W, np.float32)
+    assert g.shape == (C,) and a.shape == (C,) and w.shape[1] == C
+    theta = ctypes.c_float(0.0)
+    losses = np.empty(P, np.float64)
+    _check(_lib.qllm_search_theta(_dp(calib_x), _xdtype(calib_x), T, C, _hp(g), None if b is None else _hp(b), ln_eps,
+                                  _hp(a), _hp(w), w.shape[0], a_bits, w_bits, P, ctypes.addressof(theta),
+                                  _hp(losses), _stream(stream)))
+    return float(theta.value), losses
 
 
 def qllm_validate_map(map_ptr, map_src, C):
