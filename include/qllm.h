@@ -74,7 +74,10 @@ extern "C" {
  *                                   alpha = |value| (1 if the value is 0).
  *
  *  x         device, [M][C] row-major, float32 (x_dtype = QLLM_F32) or bfloat16 (QLLM_BF16)
- *  ln_gamma  device float[C];  ln_beta device float[C] or NULL (= 0)
+ *  ln_gamma  device float[C];  ln_beta device float[C] or NULL (= 0).  ln_gamma = NULL (then ln_beta
+ *            = NULL too): no LayerNorm, x already is the linear layer's input -- the case of Appendix B,
+ *            where a preceding linear layer absorbed the map (qllm_fold_previous) and the map passed
+ *            here is the identity.  This mode runs on the shape-agnostic kernel.
  *  map_ptr   device int32[C+1], map_src device int32[nnz], map_coef device float[nnz];
  *            rows non-empty, 0 <= src < C.  The map is NOT validated on the device: use
  *            qllm_validate_map on the host copy if it does not come from the builder.
@@ -207,6 +210,15 @@ int qllm_reassembly_weights(const qllm_reassembly_t* h, const uint8_t** w_codes,
 /* stats[0] = E (channels added by disassembly = merges done), stats[1] = rows with more than
  * one member, stats[2] = matching rounds, stats[3] = C, stats[4] = N, stats[5] = w_bits */
 int qllm_reassembly_stats(const qllm_reassembly_t* h, int64_t stats[6]);
+
+/* Appendix B: when the layer in front of the quantized layer is itself linear, the map needs no run-time
+ * kernel: it is applied once to that layer's output channels.  W_prev is HOST float[C_src][C_in] (output
+ * channel major; C_src = number of source channels the map refers to), bias_prev HOST float[C_src] or NULL;
+ * W_out HOST float[C][C_in] and bias_out HOST float[C] receive  row c = sum_j coef_j * row src_j  (a
+ * sub-channel becomes the source row divided by T, a merged channel the mean of its members' rows), summed in
+ * double in entry order.  x W_out^T + bias_out then equals the map applied to x W_prev^T + bias_prev. */
+int qllm_fold_previous(const int32_t* map_ptr, const int32_t* map_src, const float* map_coef, int C,
+                       const float* W_prev, const float* bias_prev, int C_in, float* W_out, float* bias_out);
 
 /* Host-side structural check of a map: ptr[0] = 0, rows non-empty and monotone, 0 <= src < C. */
 int qllm_validate_map(const int32_t* map_ptr, const int32_t* map_src, int C, int64_t nnz);

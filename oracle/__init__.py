@@ -274,3 +274,24 @@ def search_theta(xcal, gamma, beta, eps, W, absmax, a_bits, w_bits, P):
     losses = np.array([reassembly_loss(xcal, gamma, beta, eps, W, absmax, float(t), a_bits, w_bits) for t in grid])
     best = int(np.argmin(losses))          # first occurrence: Algorithm 1 updates only on a strictly smaller loss
     return float(grid[best]), losses
+
+
+# ---------------------------------------------------------------------------
+# Appendix B: the map folded into a preceding linear layer (plain numpy, fp64).
+# ---------------------------------------------------------------------------
+def fold_previous(W_prev, bias_prev, ptr, src, coef):
+    """Row c of the result = sum_j coef_j * row src_j of W_prev [C_src][C_in] (and of its bias): the
+    preceding layer's output channels duplicated with 1/T (disassembly) and averaged (assembly).
+    Returns (W_out float32 [C][C_in], bias_out float32 [C] or None), sums taken in fp64 in entry order."""
+    W = np.asarray(W_prev, np.float32).astype(np.float64)
+    b = None if bias_prev is None else np.asarray(bias_prev, np.float32).astype(np.float64)
+    C = len(ptr) - 1
+    out = np.zeros((C, W.shape[1]), np.float64)
+    bout = None if b is None else np.zeros(C, np.float64)
+    for c in range(C):
+        for j in range(int(ptr[c]), int(ptr[c + 1])):
+            cf = float(np.float32(coef[j]))
+            out[c] += cf * W[int(src[j])]
+            if b is not None:
+                bout[c] += cf * b[int(src[j])]
+    return out.astype(np.float32), None if bout is None else bout.astype(np.float32)

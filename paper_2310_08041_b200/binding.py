@@ -26,7 +26,7 @@ QLLM_F32, QLLM_BF16 = 0, 1
 EXPORTS = [
     "qllm_reassemble_quant", "qllm_qgemm", "qllm_qgemm_noalloc", "qllm_qgemm_acc", "qllm_calib_absmax",
     "qllm_build_reassembly", "qllm_free_reassembly", "qllm_reassembly_map",
-    "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map",
+    "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map", "qllm_fold_previous",
     "qllm_theta_percentile", "qllm_theta_for_extra", "qllm_search_theta",
     "qllm_layer_create", "qllm_layer_destroy", "qllm_layer_forward", "qllm_layer_forward_host",
     "qllm_layer_reassemble_quant", "qllm_layer_qgemm",
@@ -57,6 +57,7 @@ _lib.qllm_validate_map.argtypes = [_vp, _vp, _i, _i64]
 _lib.qllm_theta_percentile.argtypes = [_vp, _i, _d]
 _lib.qllm_theta_percentile.restype = _f
 _lib.qllm_search_theta.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _vp]
+_lib.qllm_fold_previous.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _vp, _vp]
 _lib.qllm_theta_for_extra.argtypes = [_vp, _i, _i]
 _lib.qllm_theta_for_extra.restype = _f
 _lib.qllm_layer_create.argtypes = [_vp, _vp, _vp, _f, _vp, _i, _i, _i, _i64, ctypes.POINTER(_vp)]
@@ -195,6 +196,19 @@ def qllm_search_theta(calib_x, ln_gamma, ln_beta, absmax, W, a_bits, w_bits, P, 
                                   _hp(a), _hp(w), w.shape[0], a_bits, w_bits, P, ctypes.addressof(theta),
                                   _hp(losses), _stream(stream)))
     return float(theta.value), losses
+
+
+def qllm_fold_previous(map_ptr, map_src, map_coef, W_prev, bias_prev=None):
+    """Appendix B: the map applied to the preceding linear layer's output channels (host).  Returns (W_out, bias_out)."""
+    p = np.ascontiguousarray(map_ptr, np.int32); s = np.ascontiguousarray(map_src, np.int32)
+    c = np.ascontiguousarray(map_coef, np.float32); w = np.ascontiguousarray(W_prev, np.float32)
+    C, C_in = p.shape[0] - 1, w.shape[1]
+    b = None if bias_prev is None else np.ascontiguousarray(bias_prev, np.float32)
+    out = np.empty((C, C_in), np.float32)
+    bout = None if b is None else np.empty(C, np.float32)
+    _check(_lib.qllm_fold_previous(_hp(p), _hp(s), _hp(c), C, _hp(w), None if b is None else _hp(b), C_in, _hp(out),
+                                   None if bout is None else _hp(bout)))
+    return out, bout
 
 
 def qllm_validate_map(map_ptr, map_src, C):

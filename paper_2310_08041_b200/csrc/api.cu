@@ -209,8 +209,8 @@ static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const 
     if (!dtype_ok(x_dtype)) return QLLM_ERR_DTYPE;
     if (M < 0 || C <= 0 || C > 49152 || (bits == 4 && (C & 1))) return QLLM_ERR_SHAPE;
     if (M == 0) return QLLM_OK;
-    if (!x || !ln_gamma || !map_ptr || !map_src || !map_coef || !codes || !a_scale || !a_zero)
-        return QLLM_ERR_NULL;
+    if (!x || !map_ptr || !map_src || !map_coef || !codes || !a_scale || !a_zero) return QLLM_ERR_NULL;
+    if (!ln_gamma && ln_beta) return QLLM_ERR_NULL;        // no LayerNorm means neither parameter
     if (!aligned16(x) || !aligned16(codes)) return QLLM_ERR_ALIGN;
     return launch_reassemble_quant(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, map_ptr, map_src,
                                    map_coef, bits, map_image, codes, a_scale, a_zero, a_rowsum,

@@ -280,6 +280,32 @@ int qllm_reassembly_stats(const qllm_reassembly_t* h, int64_t stats[6]) {
     return QLLM_OK;
 }
 
+int qllm_fold_previous(const int32_t* map_ptr, const int32_t* map_src, const float* map_coef, int C,
+                       const float* W_prev, const float* bias_prev, int C_in, float* W_out, float* bias_out) {
+    if (!map_ptr || !map_src || !map_coef || !W_prev || !W_out) return QLLM_ERR_NULL;
+    if (C <= 0 || C_in <= 0) return QLLM_ERR_SHAPE;
+    if (bias_prev && !bias_out) return QLLM_ERR_NULL;
+    const int rc = qllm_validate_map(map_ptr, map_src, C, map_ptr[C]);
+    if (rc != QLLM_OK) return rc;
+    // output channel c of the preceding layer = sum_j coef_j * (its output channel src_j): Appendix B's
+    // duplication with 1/T for sub-channels and the mean for merged channels, in one pass over the map
+    std::vector<double> acc(static_cast<size_t>(C_in));
+    for (int c = 0; c < C; ++c) {
+        std::fill(acc.begin(), acc.end(), 0.0);
+        double b = 0.0;
+        for (int j = map_ptr[c]; j < map_ptr[c + 1]; ++j) {
+            const double cf = double(map_coef[j]);
+            const float* row = W_prev + size_t(map_src[j]) * C_in;
+            for (int k = 0; k < C_in; ++k) acc[k] += cf * double(row[k]);
+            if (bias_prev) b += cf * double(bias_prev[map_src[j]]);
+        }
+        float* out = W_out + size_t(c) * C_in;
+        for (int k = 0; k < C_in; ++k) out[k] = float(acc[k]);
+        if (bias_prev) bias_out[c] = float(b);
+    }
+    return QLLM_OK;
+}
+
 int qllm_validate_map(const int32_t* map_ptr, const int32_t* map_src, int C, int64_t nnz) {
     if (!map_ptr || !map_src) return QLLM_ERR_NULL;
     if (C <= 0 || nnz < C) return QLLM_ERR_MAP;

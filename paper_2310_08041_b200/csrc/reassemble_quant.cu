@@ -781,7 +781,7 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
                             const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
                             float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes, int slots_known,
                             bool share_sm) {
-    if (!warp_kernel_serves(C)) {
+    if (!warp_kernel_serves(C) || !gamma) {              // no LayerNorm: the shape-agnostic kernel
         if (byte_lanes && bits == 4) return QLLM_ERR_UNSUPPORTED;
         return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
                                                a_scale, a_zero, a_rowsum, st);

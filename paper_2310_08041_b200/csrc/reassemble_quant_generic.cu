@@ -26,9 +26,16 @@ __device__ __forceinline__ float load_as_float<__nv_bfloat16>(const __nv_bfloat1
 }
 
 // LayerNorm of one row into shared memory y[0..C).  All threads of the CTA take part.
+// gamma == nullptr: no normalisation, the row is copied as it is (the caller's input already is the
+// linear layer's input, Appendix B).
 template <typename XT>
 __device__ void layernorm_row(const XT* __restrict__ xrow, int C, const float* __restrict__ gamma,
                               const float* __restrict__ beta, float eps, float* y, float* red) {
+    if (!gamma) {
+        for (int k = threadIdx.x; k < C; k += blockDim.x) y[k] = load_as_float<XT>(xrow, k);
+        __syncthreads();
+        return;
+    }
     float s = 0.f;
     for (int k = threadIdx.x; k < C; k += blockDim.x) {
         float v = load_as_float<XT>(xrow, k);

@@ -31,7 +31,7 @@ def run_reassemble_quant(x_np, gamma, beta, eps, ptr, src, coef, bits, want_rows
     a_scale = torch.full((M,), -1.0, dtype=torch.float32, device=DEV)
     a_zero = torch.full((M,), -1e9, dtype=torch.float32, device=DEV)
     a_rowsum = torch.full((M,), -7, dtype=torch.int32, device=DEV) if want_rowsum else None
-    B.qllm_reassemble_quant(x, dev(gamma), None if beta is None else dev(beta), dev(ptr), dev(src), dev(coef),
+    B.qllm_reassemble_quant(x, None if gamma is None else dev(gamma), None if beta is None else dev(beta), dev(ptr), dev(src), dev(coef),
                             bits, codes, a_scale, a_zero, a_rowsum, ln_eps=eps)
     torch.cuda.synchronize()
     stored = codes.cpu().numpy()

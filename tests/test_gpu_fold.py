@@ -1,0 +1,41 @@
+"""Appendix B on the product path: the host fold against the oracle's, and the run-time half (per-token
+quantization without LayerNorm on an identity map) against the oracle."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2310_08041_b200 import synth
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def test_fold_previous_matches_oracle_and_quantizes_without_layernorm():
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    cfg = synth.CONFIGS["c1"].scaled(M=40, K=256)
+    L = parity.oracle_layer(cfg, with_weights=False)
+    rng = np.random.default_rng(9)
+    C_in = 96
+    Wp = (0.3 * rng.standard_normal((cfg.K, C_in))).astype(np.float32)     # preceding layer: C_in -> K channels
+    bp = (0.1 * rng.standard_normal(cfg.K)).astype(np.float32)
+    ref_W, ref_b = oracle.fold_previous(Wp, bp, L["ptr"], L["src"], L["coef"])
+    W2, b2 = B.qllm_fold_previous(L["ptr"], L["src"], L["coef"], Wp, bp)
+    assert np.array_equal(W2, ref_W) and np.array_equal(b2, ref_b)
+    # run time: the folded layer's output already is the reassembled activation; quantize it as it is
+    X = rng.standard_normal((cfg.M, C_in)).astype(np.float32)
+    X[:, 5] *= 40.0
+    xr = (X.astype(np.float64) @ W2.astype(np.float64).T + b2).astype(np.float32)
+    C = cfg.K
+    ident = (np.arange(C + 1, dtype=np.int32), np.arange(C, dtype=np.int32), np.ones(C, np.float32))
+    for bits in (4, 8):
+        got = G.run_reassemble_quant(xr, None, None, 0.0, *ident, bits)
+        ref = oracle.quant_rows(xr.astype(np.float64), bits, want_pre=True)
+        ref["xr"] = xr
+        old = parity.FLIP_BAND
+        parity.FLIP_BAND = old * (17 if bits == 8 else 1)
+        try:
+            parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref, bits)
+        finally:
+            parity.FLIP_BAND = old

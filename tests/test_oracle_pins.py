@@ -433,3 +433,31 @@ def test_search_theta_is_the_first_minimum_of_the_grid_losses():
         assert losses[p] == oracle.reassembly_loss(x, gamma, None, 1e-5, W, absmax, float(grid[p]), 4, 4)
     # splitting the outlier channels helps on this input: some interior threshold beats "no reassembly"
     assert losses[best] < losses[-1]
+
+
+# ---------------------------------------------------------------------------
+# Appendix B: reassembly folded into a preceding linear layer
+# ---------------------------------------------------------------------------
+def test_fold_previous_closed_forms_and_function_preservation():
+    """Appendix B's two rules on a hand-made map (channel 1 split in T = 3, channels 2 and 4 merged), then
+    the defining property: the folded layer's output equals the map applied to the original output."""
+    rng = np.random.default_rng(5)
+    C_src, C_in = 5, 7
+    Wp = rng.standard_normal((C_src, C_in)).astype(np.float32)
+    bp = rng.standard_normal(C_src).astype(np.float32)
+    third = np.float32(1.0 / 3.0)
+    rows = [[(0, 1.0)], [(1, third)], [(1, third)], [(1, third)], [(2, 0.5), (4, 0.5)]]   # 5 rows: 3 stays out
+    ptr = np.array([0, 1, 2, 3, 4, 6], np.int32)
+    src = np.array([s for r in rows for s, _ in r], np.int32)
+    coef = np.array([c for r in rows for _, c in r], np.float32)
+    Wo, bo = oracle.fold_previous(Wp, bp, ptr, src, coef)
+    assert np.array_equal(Wo[0], Wp[0])                                             # untouched channel
+    for c in (1, 2, 3):                                                             # W / T
+        np.testing.assert_allclose(Wo[c], Wp[1].astype(np.float64) * float(third), rtol=1e-7)
+    np.testing.assert_allclose(Wo[4], (Wp[2].astype(np.float64) + Wp[4]) / 2, rtol=1e-7)   # (W_i + W_j) / 2
+    np.testing.assert_allclose(bo[4], (float(bp[2]) + float(bp[4])) / 2, rtol=1e-6)
+    X = rng.standard_normal((9, C_in))
+    y_prev = X @ Wp.astype(np.float64).T + bp
+    want = oracle.map_apply(y_prev, ptr, src, coef)
+    got = X @ Wo.astype(np.float64).T + bo
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-6)                        # fp32 storage of the rows
