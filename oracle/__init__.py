@@ -204,18 +204,41 @@ class Infeasible(Exception):
     pass
 
 
-def build_map(absmax, theta):
-    """Returns (ptr i32[C+1], src i32[nnz], coef f32[nnz], stats dict)."""
+class NeedsMoreRounds(Exception):
+    """Eq. 5 distances are defined between undivided channels: one matching round only."""
+
+
+def channel_distance(y, W):
+    """Eq. 5 table D[i][j] = 1/4 ||y_i - y_j||^2 ||W_i - W_j||^2 (float32, defined order).  y [T][C], W [N][C]."""
+    y = _c(y, np.float32); W = _c(W, np.float32)
+    T, C = y.shape
+    N = W.shape[0]
+    assert W.shape[1] == C
+    D = np.empty((C, C), np.float32)
+    lib().orc_channel_distance(_p(y), ctypes.c_int64(T), _p(W), ctypes.c_int(N), ctypes.c_int(C), _p(D))
+    return D
+
+
+def build_map(absmax, theta, dist=None):
+    """Returns (ptr i32[C+1], src i32[nnz], coef f32[nnz], stats dict).  dist: optional Eq. 5 table [C][C]."""
     a = _c(absmax, np.float32)
     C = a.shape[0]
     E = extra_channels(a, theta)
     cap = C + E
     ptr = np.empty(C + 1, np.int32); src = np.empty(cap, np.int32); coef = np.empty(cap, np.float32)
     stats = np.zeros(3, np.int64)
-    rc = lib().orc_build_map(_p(a), ctypes.c_int(C), ctypes.c_float(theta), _p(ptr), _p(src), _p(coef),
-                             ctypes.c_int64(cap), _p(stats))
+    if dist is None:
+        rc = lib().orc_build_map(_p(a), ctypes.c_int(C), ctypes.c_float(theta), _p(ptr), _p(src), _p(coef),
+                                 ctypes.c_int64(cap), _p(stats))
+    else:
+        d = _c(dist, np.float32)
+        assert d.shape == (C, C)
+        rc = lib().orc_build_map_dist(_p(a), ctypes.c_int(C), ctypes.c_float(theta), _p(d), _p(ptr), _p(src), _p(coef),
+                                      ctypes.c_int64(cap), _p(stats))
     if rc == -1:
         raise Infeasible()
+    if rc == -4:
+        raise NeedsMoreRounds()
     assert rc == 0, rc
     nnz = int(ptr[C])
     return ptr, src[:nnz].copy(), coef[:nnz].copy(), dict(E=int(stats[0]), merged_rows=int(stats[1]),

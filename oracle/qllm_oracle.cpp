@@ -351,8 +351,12 @@ float orc_theta_for_extra(const float* absmax, int C, int extra) {
 // the caller's buffers are too small (nnz_cap).
 // stats[0] = E, stats[1] = rows with more than one member, stats[2] = rounds.
 // ---------------------------------------------------------------------------
-int orc_build_map(const float* absmax, int C, float theta, int32_t* ptr, int32_t* src,
-                  float* coef, int64_t nnz_cap, int64_t* stats) {
+// dist: optional C x C table of pairwise channel distances (Eq. 5, see orc_channel_distance).  Without it the
+// distance between two entries is |m_a - m_b|.  With it the distance between two undivided channels is
+// dist[a][b]; a second matching round would need distances between merged sets, which Eq. 5 does not define:
+// -4 is returned instead.
+static int build_map_impl(const float* absmax, int C, float theta, const float* dist, int32_t* ptr, int32_t* src,
+                          float* coef, int64_t nnz_cap, int64_t* stats) {
     if (!(theta > 0.f)) return -3;
     std::vector<Entry> list;
     int64_t E = 0;
@@ -372,6 +376,7 @@ int orc_build_map(const float* absmax, int C, float theta, int32_t* ptr, int32_t
     int64_t need = E;
     int rounds = 0;
     while (need > 0) {
+        if (dist && rounds > 0) return -4;
         std::vector<int> A, B;
         for (int p = 0; p < static_cast<int>(list.size()); ++p) {
             if (list[p].is_sub) continue;
@@ -384,7 +389,8 @@ int orc_build_map(const float* absmax, int C, float theta, int32_t* ptr, int32_t
             double best = std::numeric_limits<double>::infinity();
             int bb = -1;
             for (int b : B) {
-                double d = std::fabs(list[a].m - list[b].m);
+                double d = dist ? static_cast<double>(dist[static_cast<int64_t>(list[a].members[0]) * C + list[b].members[0]])
+                                : std::fabs(list[a].m - list[b].m);
                 if (d < best) { best = d; bb = b; }   // B ascending: first minimum = lowest position
             }
             edges.push_back({best, a, bb});
@@ -429,6 +435,44 @@ int orc_build_map(const float* absmax, int C, float theta, int32_t* ptr, int32_t
     ptr[C] = static_cast<int32_t>(nnz);
     if (stats) { stats[0] = E; stats[1] = multi; stats[2] = rounds; }
     return 0;
+}
+
+int orc_build_map(const float* absmax, int C, float theta, int32_t* ptr, int32_t* src,
+                  float* coef, int64_t nnz_cap, int64_t* stats) {
+    return build_map_impl(absmax, C, theta, nullptr, ptr, src, coef, nnz_cap, stats);
+}
+
+// The same builder with the distance of Eq. 5 between undivided channels, given as a C x C table.
+int orc_build_map_dist(const float* absmax, int C, float theta, const float* dist, int32_t* ptr, int32_t* src,
+                       float* coef, int64_t nnz_cap, int64_t* stats) {
+    if (!dist) return -3;
+    return build_map_impl(absmax, C, theta, dist, ptr, src, coef, nnz_cap, stats);
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 5: the output error of merging channels i and j,
+//     D(i, j) = || (x_i (W_i - W_j) + x_j (W_j - W_i)) / 2 ||_F^2 = 1/4 ||x_i - x_j||^2 ||W_i - W_j||^2,
+// x_i the column of channel i over the T calibration rows of y (the linear layer's input), W_i the
+// weights of input channel i over the N outputs.  The table decides an argmin (the nearest channel), so it
+// is computed in the precision and order the product uses: float32, rows taken in order with one fused
+// multiply-add each,   dx = fma(e, e, dx), e = y[t][i] - y[t][j];   D = (0.25f * dx) * dw.
+// y: [T][C], w: [N][C] (output channel major), D: [C][C].
+// ---------------------------------------------------------------------------
+void orc_channel_distance(const float* y, int64_t T, const float* w, int N, int C, float* D) {
+    for (int i = 0; i < C; ++i) {
+        for (int j = 0; j < C; ++j) {
+            float dx = 0.f, dw = 0.f;
+            for (int64_t t = 0; t < T; ++t) {
+                const float e = y[t * C + i] - y[t * C + j];
+                dx = std::fmaf(e, e, dx);
+            }
+            for (int n = 0; n < N; ++n) {
+                const float e = w[static_cast<int64_t>(n) * C + i] - w[static_cast<int64_t>(n) * C + j];
+                dw = std::fmaf(e, e, dw);
+            }
+            D[static_cast<int64_t>(i) * C + j] = (0.25f * dx) * dw;
+        }
+    }
 }
 
 }  // extern "C"

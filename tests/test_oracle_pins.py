@@ -461,3 +461,76 @@ def test_fold_previous_closed_forms_and_function_preservation():
     want = oracle.map_apply(y_prev, ptr, src, coef)
     got = X @ Wo.astype(np.float64).T + bo
     np.testing.assert_allclose(got, want, rtol=0, atol=1e-6)                        # fp32 storage of the rows
+
+
+# ---------------------------------------------------------------------------
+# Eq. 5: distance between channels, and the builder driven by it
+# ---------------------------------------------------------------------------
+def _eq5_case(seed=21, T=20, C=24, N=18):
+    rng = np.random.default_rng(seed)
+    y = rng.standard_normal((T, C)).astype(np.float32)
+    W = (0.2 * rng.standard_normal((N, C))).astype(np.float32)
+    return y, W
+
+
+def test_channel_distance_is_eq5_and_equals_the_error_of_the_merge():
+    y, W = _eq5_case()
+    D = oracle.channel_distance(y, W)
+    C = y.shape[1]
+    y64, W64 = y.astype(np.float64), W.astype(np.float64)
+    ref = np.array([[0.25 * ((y64[:, i] - y64[:, j]) ** 2).sum() * ((W64[:, i] - W64[:, j]) ** 2).sum()
+                     for j in range(C)] for i in range(C)])
+    np.testing.assert_allclose(D, ref, rtol=2e-5, atol=0)
+    assert np.array_equal(D, D.T) and np.all(np.diag(D) == 0)
+    # Eq. 5 is the output error of assembling the two channels (Eq. 4): build that map by hand and measure it
+    i, j = 3, 10
+    rows = [[c] for c in range(C) if c != j]
+    rows[i] = [i, j]
+    rows.append([j])                                    # keep C rows: channel j again as its own row, then drop its effect
+    ptr = np.zeros(C + 1, np.int32); ptr[1:] = np.cumsum([len(r) for r in rows])
+    src = np.array([s for r in rows for s in r], np.int32)
+    coef = np.array([1.0 / len(r) for r in rows for _ in r], np.float32)
+    xr = oracle.map_apply(y64, ptr, src, coef)[:, :C - 1]            # the C - 1 assembled channels
+    Wr = oracle.weight_transform(W, ptr, src)[:, :C - 1]
+    err = ((y64 @ W64.T - xr @ Wr.T) ** 2).sum()
+    assert abs(err - ref[i, j]) <= 1e-9 * ref[i, j]
+
+
+def test_builder_with_a_distance_table():
+    """With the table |m_i - m_j| the table-driven builder is the plain one (integer maxima keep the table exact);
+    with an Eq. 5 table it follows the brute-force statement of Appendix A steps 2-3 on that table."""
+    rng = np.random.default_rng(22)
+    C = 36
+    absmax = rng.integers(1, 9, C).astype(np.float32)
+    absmax[[4, 19]] = [40.0, 23.0]
+    theta = 9.0
+    table = np.abs(absmax[:, None] - absmax[None, :]).astype(np.float32)
+    a = oracle.build_map(absmax, theta)
+    b = oracle.build_map(absmax, theta, dist=table)
+    assert a[3]["rounds"] == 1 and all(np.array_equal(u, v) for u, v in zip(a[:3], b[:3]))
+    y, W = _eq5_case(seed=23, C=C)
+    D = oracle.channel_distance(y, W)
+    ptr, src, coef, st = oracle.build_map(absmax, theta, dist=D)
+    T = np.maximum(1, np.ceil(absmax / np.float32(theta))).astype(int)
+    pos_src = np.repeat(np.arange(C), T)
+    elig = [p for p in range(len(pos_src)) if T[pos_src[p]] == 1]
+    A = [p for p in elig if p % 2 == 0]; B = [p for p in elig if p % 2 == 1]
+    edges = []
+    for p in A:
+        d = [float(D[pos_src[p], pos_src[q]]) for q in B]
+        edges.append((min(d), p, B[int(np.argmin(d))]))
+    edges.sort()
+    kept = edges[:st["E"]]
+    merged = {}
+    for _, p, q in sorted(kept, key=lambda e: e[1]):
+        merged.setdefault(q, [pos_src[q]]).append(pos_src[p])
+    gone = {p for _, p, _ in kept}
+    rows = [merged.get(p, [pos_src[p]]) for p in range(len(pos_src)) if p not in gone]
+    assert [src[ptr[c]:ptr[c + 1]].tolist() for c in range(C)] == [list(map(int, r)) for r in rows]
+    _check_map_invariants(absmax, theta, ptr, src, coef, st)
+    # a threshold that needs a second round has no Eq. 5 reading
+    big = absmax.copy()
+    big[4] = 400.0                                      # 44 extra channels against 17 candidates per round
+    assert oracle.build_map(big, theta)[3]["rounds"] > 1
+    with pytest.raises(oracle.NeedsMoreRounds):
+        oracle.build_map(big, theta, dist=D)
