@@ -530,7 +530,7 @@ def test_builder_with_a_distance_table():
     _check_map_invariants(absmax, theta, ptr, src, coef, st)
     # a threshold that needs a second round has no Eq. 5 reading
     big = absmax.copy()
-    big[4] = 400.0                                      # 44 extra channels against 17 candidates per round
+    big[4] = 200.0                                      # 24 extra channels against 17 candidates in the first round
     assert oracle.build_map(big, theta)[3]["rounds"] > 1
     with pytest.raises(oracle.NeedsMoreRounds):
         oracle.build_map(big, theta, dist=D)
