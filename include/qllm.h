@@ -201,6 +201,27 @@ int qllm_build_reassembly(const float* calib_absmax, int C, float theta,
                           int w_bits, qllm_reassembly_t** out);
 void qllm_free_reassembly(qllm_reassembly_t* h);
 
+/* The same builder with the distance of Eq. 5 in the bipartite matching: dist is a HOST float[C][C] table,
+ * dist[i][j] = 1/4 ||y_i - y_j||^2 ||W_i - W_j||^2 over the calibration tokens (qllm_channel_distance computes it
+ * on the device).  Nearest counterpart, tie rules and edge selection are those of qllm_build_reassembly with
+ * dist[a][b] in place of |m_a - m_b|.  Eq. 5 is defined between undivided channels, so only one matching round
+ * is possible: a threshold that needs a second round returns QLLM_ERR_UNSUPPORTED. */
+int qllm_build_reassembly_eq5(const float* calib_absmax, int C, float theta, const float* dist,
+                              const float* W, int N,
+                              const float* lr_A, const float* lr_B, int r,
+                              int w_bits, qllm_reassembly_t** out);
+
+/* Build-time device helpers for that table (asynchronous on stream; all pointers DEVICE).
+ * qllm_layernorm_rows: y[t][c] = LayerNorm(x[t])[c] as float32, the linear layer's input of the calibration
+ * tokens (x [T][C] in x_dtype, ln_beta may be NULL).
+ * qllm_channel_distance: D[i][j] of Eq. 5 from y [T][C] and the layer's weights W [N][C] (output channel major,
+ * float32), D float[C][C].  The table decides an argmin, so its arithmetic is fixed: float32, rows taken in
+ * order with one fused multiply-add each (dx = fma(e, e, dx), e = y[t][i] - y[t][j]; dw likewise over W's rows),
+ * D = (0.25f * dx) * dw; the result is bit-reproducible and symmetric. */
+int qllm_layernorm_rows(const void* x, int x_dtype, int64_t T, int C, const float* ln_gamma,
+                        const float* ln_beta, float ln_eps, float* y, void* stream);
+int qllm_channel_distance(const float* y, int64_t T, const float* W, int N, int C, float* D, void* stream);
+
 /* Borrowed host pointers into the handle (valid until qllm_free_reassembly). */
 int qllm_reassembly_map(const qllm_reassembly_t* h, const int32_t** map_ptr,
                         const int32_t** map_src, const float** map_coef, int64_t* nnz);

@@ -25,7 +25,7 @@ QLLM_F32, QLLM_BF16 = 0, 1
 # every symbol include/qllm.h declares
 EXPORTS = [
     "qllm_reassemble_quant", "qllm_qgemm", "qllm_qgemm_noalloc", "qllm_qgemm_acc", "qllm_calib_absmax",
-    "qllm_build_reassembly", "qllm_free_reassembly", "qllm_reassembly_map",
+    "qllm_build_reassembly", "qllm_build_reassembly_eq5", "qllm_layernorm_rows", "qllm_channel_distance", "qllm_free_reassembly", "qllm_reassembly_map",
     "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map", "qllm_fold_previous",
     "qllm_theta_percentile", "qllm_theta_for_extra", "qllm_search_theta",
     "qllm_layer_create", "qllm_layer_destroy", "qllm_layer_forward", "qllm_layer_forward_host",
@@ -47,6 +47,9 @@ _lib.qllm_qgemm_noalloc.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
 _lib.qllm_qgemm_acc.argtypes = [_vp, _vp, _vp, _i64, _i, _i, _i, _i, _vp]
 _lib.qllm_calib_absmax.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp]
 _lib.qllm_build_reassembly.argtypes = [_vp, _i, _f, _vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(_vp)]
+_lib.qllm_build_reassembly_eq5.argtypes = [_vp, _i, _f, _vp, _vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(_vp)]
+_lib.qllm_layernorm_rows.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp]
+_lib.qllm_channel_distance.argtypes = [_vp, _i64, _vp, _i, _i, _vp, _vp]
 _lib.qllm_free_reassembly.argtypes = [_vp]
 _lib.qllm_free_reassembly.restype = None
 _lib.qllm_reassembly_map.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_i64)]
@@ -228,7 +231,7 @@ class Reassembly:
         self.free()
 
     def free(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:   # at interpreter exit the module may be gone first
             _lib.qllm_free_reassembly(self._h)
             self._h = None
 
@@ -265,7 +268,20 @@ class Reassembly:
         return codes, scale, zero, colsum
 
 
-def qllm_build_reassembly(calib_absmax, theta, W, lr_A=None, lr_B=None, w_bits=4):
+def qllm_layernorm_rows(x, ln_gamma, ln_beta, y, ln_eps=1e-5, stream=None):
+    """x, ln_gamma, ln_beta (or None), y (float32 [T][C]): device tensors."""
+    T, C = x.shape
+    _check(_lib.qllm_layernorm_rows(_dp(x), _xdtype(x), T, C, _dp(ln_gamma), _dp(ln_beta), ln_eps, _dp(y), _stream(stream)))
+
+
+def qllm_channel_distance(y, W, D, stream=None):
+    """y float32 [T][C], W float32 [N][C], D float32 [C][C]: device tensors (Eq. 5 table)."""
+    T, C = y.shape
+    _check(_lib.qllm_channel_distance(_dp(y), T, _dp(W), W.shape[0], C, _dp(D), _stream(stream)))
+
+
+def qllm_build_reassembly(calib_absmax, theta, W, lr_A=None, lr_B=None, w_bits=4, dist=None):
+    """dist: optional host float32 [C][C] table of Eq. 5 distances (then qllm_build_reassembly_eq5 is called)."""
     a = np.ascontiguousarray(calib_absmax, np.float32)
     W = np.ascontiguousarray(W, np.float32)
     N, C = W.shape
@@ -277,7 +293,13 @@ def qllm_build_reassembly(calib_absmax, theta, W, lr_A=None, lr_B=None, w_bits=4
         r = lr_A.shape[1]
         assert lr_A.shape == (C, r) and lr_B.shape == (r, N)
     h = _vp()
-    _check(_lib.qllm_build_reassembly(_hp(a), C, theta, _hp(W), N, _hp(lr_A), _hp(lr_B), r, w_bits, ctypes.byref(h)))
+    if dist is None:
+        _check(_lib.qllm_build_reassembly(_hp(a), C, theta, _hp(W), N, _hp(lr_A), _hp(lr_B), r, w_bits, ctypes.byref(h)))
+    else:
+        d = np.ascontiguousarray(dist, np.float32)
+        assert d.shape == (C, C)
+        _check(_lib.qllm_build_reassembly_eq5(_hp(a), C, theta, _hp(d), _hp(W), N, _hp(lr_A), _hp(lr_B), r, w_bits,
+                                              ctypes.byref(h)))
     return Reassembly(h, C, N)
 
 
@@ -299,7 +321,7 @@ class Layer:
         self.destroy()
 
     def destroy(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:   # at interpreter exit the module may be gone first
             _lib.qllm_layer_destroy(self._h)
             self._h = None
 

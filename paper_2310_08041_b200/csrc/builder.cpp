@@ -52,8 +52,10 @@ struct BKey {
 
 // One round of bipartite soft matching on `slots`; merges up to `need` A-slots into
 // their nearest B-slot.  Returns the number of merges done (0 = no eligible pair).
+// dist (optional): C x C table of Eq. 5 distances between undivided channels; the nearest b of an a is then
+// found by a scan over B on that table (the table has no order to search in).
 int64_t matching_round(std::vector<Slot>& slots, std::vector<int>& next_member,
-                       const float* absmax, int64_t need) {
+                       const float* absmax, int64_t need, const float* dist, int C) {
     const int L = int(slots.size());
     std::vector<int> A;
     std::vector<BKey> B;
@@ -67,7 +69,22 @@ int64_t matching_round(std::vector<Slot>& slots, std::vector<int>& next_member,
 
     struct Edge { double d; int a; int b; };
     std::vector<Edge> edges(A.size());
-    for (size_t i = 0; i < A.size(); ++i) {
+    if (dist) {
+        std::vector<int> Bpos;                            // B in list order: ties go to the lowest position
+        for (int p = 1; p < L; p += 2)
+            if (!slots[p].sub) Bpos.push_back(p);
+        for (size_t i = 0; i < A.size(); ++i) {
+            const float* row = dist + size_t(slots[A[i]].head) * size_t(C);
+            double best = std::numeric_limits<double>::infinity();
+            int best_pos = -1;
+            for (int p : Bpos) {
+                const double d = double(row[slots[p].head]);
+                if (d < best) { best = d; best_pos = p; }
+            }
+            edges[i] = {best, A[i], best_pos};
+        }
+    }
+    for (size_t i = 0; i < A.size() && !dist; ++i) {
         const int a = A[i];
         const double ma = slots[a].m;
         // first key with m >= ma
@@ -114,7 +131,7 @@ int64_t matching_round(std::vector<Slot>& slots, std::vector<int>& next_member,
     return keep;
 }
 
-int build_map(const float* absmax, int C, float theta, qllm_reassembly& h) {
+int build_map(const float* absmax, int C, float theta, const float* dist, qllm_reassembly& h) {
     std::vector<Slot> slots;
     slots.reserve(size_t(C) + 64);
     int64_t E = 0;
@@ -127,7 +144,8 @@ int build_map(const float* absmax, int C, float theta, qllm_reassembly& h) {
     std::vector<int> next_member(size_t(C), -1);
     int64_t need = E, rounds = 0;
     while (need > 0) {
-        int64_t done = matching_round(slots, next_member, absmax, need);
+        if (dist && rounds > 0) return QLLM_ERR_UNSUPPORTED;   // Eq. 5 is defined between undivided channels only
+        int64_t done = matching_round(slots, next_member, absmax, need, dist, C);
         if (done == 0) return QLLM_ERR_INFEASIBLE;
         need -= done;
         ++rounds;
@@ -224,9 +242,9 @@ void transform_and_quantize(const float* W, int N, int C, const float* lrA, cons
 
 extern "C" {
 
-int qllm_build_reassembly(const float* calib_absmax, int C, float theta, const float* W, int N,
-                          const float* lr_A, const float* lr_B, int r, int w_bits,
-                          qllm_reassembly_t** out) {
+static int build_reassembly_impl(const float* calib_absmax, int C, float theta, const float* dist, const float* W,
+                                 int N, const float* lr_A, const float* lr_B, int r, int w_bits,
+                                 qllm_reassembly_t** out) {
     if (!calib_absmax || !W || !out) return QLLM_ERR_NULL;
     if ((lr_A == nullptr) != (lr_B == nullptr)) return QLLM_ERR_NULL;
     if (C <= 0 || N <= 0 || C > 65536 || (lr_A && r <= 0)) return QLLM_ERR_SHAPE;
@@ -240,7 +258,7 @@ int qllm_build_reassembly(const float* calib_absmax, int C, float theta, const f
     h->C = C; h->N = N; h->w_bits = w_bits;
     int rc;
     try {
-        rc = build_map(calib_absmax, C, theta, *h);
+        rc = build_map(calib_absmax, C, theta, dist, *h);
         if (rc == QLLM_OK) transform_and_quantize(W, N, C, lr_A, lr_B, r, w_bits, *h);
     } catch (const std::bad_alloc&) {
         rc = QLLM_ERR_NOMEM;
@@ -248,6 +266,19 @@ int qllm_build_reassembly(const float* calib_absmax, int C, float theta, const f
     if (rc != QLLM_OK) { delete h; return rc; }
     *out = h;
     return QLLM_OK;
+}
+
+int qllm_build_reassembly(const float* calib_absmax, int C, float theta, const float* W, int N,
+                          const float* lr_A, const float* lr_B, int r, int w_bits,
+                          qllm_reassembly_t** out) {
+    return build_reassembly_impl(calib_absmax, C, theta, nullptr, W, N, lr_A, lr_B, r, w_bits, out);
+}
+
+int qllm_build_reassembly_eq5(const float* calib_absmax, int C, float theta, const float* dist, const float* W,
+                              int N, const float* lr_A, const float* lr_B, int r, int w_bits,
+                              qllm_reassembly_t** out) {
+    if (!dist) return QLLM_ERR_NULL;
+    return build_reassembly_impl(calib_absmax, C, theta, dist, W, N, lr_A, lr_B, r, w_bits, out);
 }
 
 void qllm_free_reassembly(qllm_reassembly_t* h) { delete h; }

@@ -83,6 +83,9 @@ int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C
                                     const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                                     const float* coef, int bits, uint8_t* codes, float* a_scale,
                                     float* a_zero, int32_t* a_rowsum, cudaStream_t st);
+// y[t][c] = LayerNorm(x[t])[c] in fp32 (build-time helper)
+int launch_layernorm_rows(const void* x, int x_dtype, int64_t T, int C, const float* gamma, const float* beta,
+                          float eps, float* y, cudaStream_t st);
 int launch_calib_absmax(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                         const float* beta, float eps, float* absmax, cudaStream_t st);
 int launch_expand_codes(const uint8_t* packed, int64_t rows, int K, uint8_t* bytes, cudaStream_t st);

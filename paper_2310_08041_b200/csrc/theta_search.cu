@@ -19,29 +19,6 @@ namespace qllm {
 
 namespace {
 
-// y[t][c] = LayerNorm(x[t])[c] in fp32; one CTA per token row.
-template <typename XT>
-__global__ void __launch_bounds__(256)
-layernorm_rows_kernel(const XT* __restrict__ x, int C, const float* __restrict__ gamma, const float* __restrict__ beta,
-                      float eps, float* __restrict__ y) {
-    __shared__ float red[32];
-    const XT* xr = x + size_t(blockIdx.x) * C;
-    float* yr = y + size_t(blockIdx.x) * C;
-    float s = 0.f;
-    for (int c = threadIdx.x; c < C; c += blockDim.x) s += float(xr[c]);
-    const float mean = block_sum(s, red) / float(C);
-    float sq = 0.f;
-    for (int c = threadIdx.x; c < C; c += blockDim.x) {
-        const float d = float(xr[c]) - mean;
-        sq = fmaf(d, d, sq);
-    }
-    const float rstd = rsqrtf(block_sum(sq, red) / float(C) + eps);
-    for (int c = threadIdx.x; c < C; c += blockDim.x) {
-        const float v = (float(xr[c]) - mean) * rstd * gamma[c];
-        yr[c] = beta ? v + beta[c] : v;
-    }
-}
-
 // out[t][n] = sum_c y[t][c] * w[n][c]; 64 x 64 tiles, 16 channels per step, 4 x 4 outputs per thread.
 __global__ void __launch_bounds__(256)
 dense_ref_kernel(const float* __restrict__ y, const float* __restrict__ w, int T, int N, int C, float* __restrict__ out) {
@@ -133,15 +110,8 @@ extern "C" int qllm_search_theta(const void* calib_x, int x_dtype, int64_t T, in
     QLLM_CUDA_TRY(cudaMemcpyAsync(d_gamma.p, ln_gamma, size_t(C) * 4, cudaMemcpyHostToDevice, st));
     if (ln_beta) QLLM_CUDA_TRY(cudaMemcpyAsync(d_beta.p, ln_beta, size_t(C) * 4, cudaMemcpyHostToDevice, st));
     QLLM_CUDA_TRY(cudaMemcpyAsync(d_w.p, W, size_t(N) * C * 4, cudaMemcpyHostToDevice, st));
-    if (x_dtype == QLLM_BF16)
-        layernorm_rows_kernel<__nv_bfloat16><<<unsigned(T), 256, 0, st>>>(
-            static_cast<const __nv_bfloat16*>(calib_x), C, static_cast<const float*>(d_gamma.p),
-            static_cast<const float*>(d_beta.p), ln_eps, static_cast<float*>(d_y.p));
-    else
-        layernorm_rows_kernel<float><<<unsigned(T), 256, 0, st>>>(
-            static_cast<const float*>(calib_x), C, static_cast<const float*>(d_gamma.p),
-            static_cast<const float*>(d_beta.p), ln_eps, static_cast<float*>(d_y.p));
-    rc = after_launch();
+    rc = launch_layernorm_rows(calib_x, x_dtype, T, C, static_cast<const float*>(d_gamma.p),
+                               static_cast<const float*>(d_beta.p), ln_eps, static_cast<float*>(d_y.p), st);
     if (rc != QLLM_OK) return rc;
     dense_ref_kernel<<<dim3(unsigned((N + 63) / 64), unsigned((T + 63) / 64)), 256, 0, st>>>(
         static_cast<const float*>(d_y.p), static_cast<const float*>(d_w.p), int(T), N, C, static_cast<float*>(d_ref.p));

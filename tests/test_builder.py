@@ -104,3 +104,32 @@ def test_theta_helpers_match():
     for extra in (1, 8, 50):
         assert B.qllm_theta_for_extra(a, extra) == oracle.theta_for_extra(a, extra)
     assert B.qllm_theta_for_extra(np.array([1.0, 1.0], np.float32), 1) == 0.0   # empty interval
+
+
+def test_builder_with_eq5_table_matches_oracle():
+    """Host builder driven by an Eq. 5 distance table (here the oracle's table: the device kernel that makes it
+    is checked bit for bit in the GPU tests) against the oracle's table-driven builder."""
+    cfg = synth.CONFIGS["c2"].scaled(M=32, K=256, N=48, n_outlier=4, calib_tokens=24)
+    g, b = synth.layernorm_params(cfg)
+    y = oracle.layernorm(synth.calibration_tokens(cfg), g, b, cfg.ln_eps).astype(np.float32)
+    absmax = oracle.channel_absmax(y)
+    W = synth.weights(cfg)
+    D = oracle.channel_distance(y, W)
+    theta = oracle.theta_percentile(absmax, 0.97)
+    ptr, src, coef, st = oracle.build_map(absmax, theta, dist=D)
+    assert st["E"] > 0 and st["rounds"] == 1
+    plain = oracle.build_map(absmax, theta)
+    assert not np.array_equal(plain[1], src)             # the Eq. 5 table picks other partners than |m_a - m_b|
+    h = B.qllm_build_reassembly(absmax, theta, W, w_bits=4, dist=D)
+    p2, s2, c2 = h.map()
+    assert np.array_equal(p2, ptr) and np.array_equal(s2, src) and np.array_equal(c2, coef)
+    ref_w = oracle.prepare_weights(W, ptr, src, 4)
+    wc, ws, wz, wcs = h.weights()
+    assert np.array_equal(wc, oracle.pack4(ref_w["codes"])) and np.array_equal(ws, ref_w["scale"])
+    # one round only: a threshold that needs two is refused
+    big = absmax.copy()
+    big[int(np.argmax(absmax))] *= 60.0
+    with pytest.raises(oracle.NeedsMoreRounds):
+        oracle.build_map(big, theta, dist=D)
+    with pytest.raises(B.QllmError):
+        B.qllm_build_reassembly(big, theta, W, w_bits=4, dist=D)
