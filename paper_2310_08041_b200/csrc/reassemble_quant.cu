@@ -34,6 +34,7 @@ namespace {
 
 constexpr int kSlotCap = 2048;                 // virtual slots an image can describe
 constexpr int kInline = 4;                     // entries held inside a slot record
+constexpr int kLongCap = 512;                  // entries of longer rows kept as (position, weight) pairs
 constexpr int kMaxWarps = 16;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
@@ -89,15 +90,23 @@ __device__ __forceinline__ void prefetch_l2(const void* p) {
 //   olo, ohi uint32[C/8][4]  the positions again as byte offsets (4 * idx), in the weights' layout
 //   vrec uint4[kSlotCap][2]  slot s: {pos0 | pos1 << 16, pos2 | pos3 << 16, w0, w1}, {w2, w3, n, 0}
 //                            for n <= kInline entries; {first CSR entry, -, -, -}, {-, -, n, 0} otherwise
-//   head int[4]         [0] = slots handed out (more than kSlotCap: the map does not fit)
+//                            for n <= kInline entries; {0, 0, 0, 0}, {first entry in lent, 0, n, 1} for a longer
+//                            row whose entries fit lent; {0, 0, 0, 0}, {first CSR entry, 0, n, 0} otherwise (the
+//                            inline fields of such a record are harmless when evaluated: positions 0)
+//   lent uint2[kLongCap]     entries of the longer rows: {position, weight bits}
+//   head int[4]         [0] = slots handed out (more than kSlotCap: the map does not fit), [1] = entries handed
+//                       out in lent, [2] = rows longer than kInline
 struct WarpImage {
     uint16_t* idx;
     float *wlo, *whi, *blo, *bhi;
     uint32_t *olo, *ohi;
     uint4* vrec;
+    uint2* lent;
     int* head;
 };
-__host__ __device__ inline size_t warp_image_bytes(int C) { return size_t(C) * 14 + size_t(kSlotCap) * 32 + 16; }
+__host__ __device__ inline size_t warp_image_bytes(int C) {
+    return size_t(C) * 14 + size_t(kSlotCap) * 32 + size_t(kLongCap) * 8 + 16;
+}
 __host__ __device__ inline WarpImage warp_image_at(void* base, int C) {
     WarpImage im;
     uint8_t* b = static_cast<uint8_t*>(base);
@@ -109,7 +118,8 @@ __host__ __device__ inline WarpImage warp_image_at(void* base, int C) {
     im.olo = reinterpret_cast<uint32_t*>(im.bhi + C / 2);
     im.ohi = im.olo + C / 2;
     im.vrec = reinterpret_cast<uint4*>(im.ohi + C / 2);
-    im.head = reinterpret_cast<int*>(im.vrec + 2 * size_t(kSlotCap));
+    im.lent = reinterpret_cast<uint2*>(im.vrec + 2 * size_t(kSlotCap));
+    im.head = reinterpret_cast<int*>(im.lent + kLongCap);
     return im;
 }
 
@@ -143,8 +153,20 @@ compile_map_warp_kernel(int C, const float* __restrict__ gamma, const float* __r
                                              __float_as_uint(ww[1]));
                 im.vrec[2 * vi + 1] = make_uint4(__float_as_uint(ww[2]), __float_as_uint(ww[3]), uint32_t(n), 0u);
             } else {
-                im.vrec[2 * vi] = make_uint4(uint32_t(j0), 0u, 0u, 0u);
-                im.vrec[2 * vi + 1] = make_uint4(0u, 0u, uint32_t(n), 0u);
+                const int first = atomicAdd(im.head + 1, n);
+                if (first + n <= kLongCap) {              // entries as (position, weight) pairs for shared memory
+                    for (int e = 0; e < n; ++e) {
+                        const int sj = __ldg(src + j0 + e);
+                        im.lent[first + e] = make_uint2(uint32_t(dplane(sj, C)),
+                                                        __float_as_uint(__ldg(coef + j0 + e) * __ldg(gamma + sj)));
+                    }
+                    im.vrec[2 * vi] = make_uint4(0u, 0u, 0u, 0u);
+                    im.vrec[2 * vi + 1] = make_uint4(uint32_t(first), 0u, uint32_t(n), 1u);
+                } else {                                  // walks the CSR arrays at run time
+                    im.vrec[2 * vi] = make_uint4(0u, 0u, 0u, 0u);
+                    im.vrec[2 * vi + 1] = make_uint4(uint32_t(j0), 0u, uint32_t(n), 0u);
+                }
+                atomicAdd(im.head + 2, 1);                // number of longer rows
             }
             pos = uint32_t(C + vi);
             w = 1.0f;
@@ -190,6 +212,16 @@ __device__ __forceinline__ float csr_row(const RawMap& rm, const float* d, int C
     for (int j = j0; j < j0 + n; ++j) {
         const int sj = __ldg(rm.src + j);
         e = fmaf(__ldg(rm.coef + j) * __ldg(rm.gamma + sj), d[dplane(sj, C)], e);
+    }
+    return e;
+}
+
+// sum of a longer row's entries kept as (position, weight) pairs
+__device__ __forceinline__ float pair_row(const uint2* ent, const float* d, int first, int n) {
+    float e = 0.f;
+    for (int k = 0; k < n; ++k) {
+        const uint2 pw = ent[first + k];
+        e = fmaf(__uint_as_float(pw.y), d[pw.x], e);
     }
     return e;
 }
@@ -297,8 +329,10 @@ reassemble_quant_warp(const XT* __restrict__ x, int64_t M, int C, float eps, int
                     e = fmaf(__uint_as_float(r1.x), d[r0.y & 0xFFFFu], e);
                     if (r1.z > 3u) e = fmaf(__uint_as_float(r1.y), d[r0.y >> 16], e);
                 }
+            } else if (r1.w) {
+                e = pair_row(im.lent, d, int(r1.x), int(r1.z));
             } else {
-                e = csr_row(rm, d, C, int(r0.x), int(r1.z));
+                e = csr_row(rm, d, C, int(r1.x), int(r1.z));
             }
             d[C + vi] = e;
         }
@@ -432,7 +466,8 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
     uint32_t* s_offB = s_offA + C / 2;
     float* s_ex = reinterpret_cast<float*>(s_offB + C / 2);             // [MAXW / G][8 G] exchange words per token slot
     uint4* s_vrec = reinterpret_cast<uint4*>(s_ex + (MAXW / G) * 8 * G);   // [row_words - C][2] slot records
-    float* rows = reinterpret_cast<float*>(s_vrec + 2 * size_t(row_words - C));
+    uint2* s_lent = reinterpret_cast<uint2*>(s_vrec + 2 * size_t(row_words - C));   // [kLongCap] entries of longer rows
+    float* rows = reinterpret_cast<float*>(s_lent + kLongCap);
 
     const int lane = threadIdx.x & 31;
     const int warp = __shfl_sync(0xffffffffu, int(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
@@ -450,11 +485,14 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
         const uint4* go = reinterpret_cast<const uint4*>(im.olo);       // olo | ohi back to back
         for (int i = threadIdx.x; i < 4 * C / 16; i += blockDim.x) cp_async16(reinterpret_cast<uint4*>(s_offA) + i, go + i);
         for (int i = threadIdx.x; i < 2 * (row_words - C); i += blockDim.x) cp_async16(s_vrec + i, im.vrec + i);
+        for (int i = threadIdx.x; i < kLongCap / 2; i += blockDim.x)
+            cp_async16(reinterpret_cast<uint4*>(s_lent) + i, reinterpret_cast<const uint4*>(im.lent) + i);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
     const int slots_total = __ldg(im.head);
     const bool slow = slots_total > row_words - C;         // uniform over the grid: walk the CSR arrays
     const int nslots = slow ? 0 : slots_total;
+    const int nlong = __ldg(im.head + 2);                  // rows longer than a slot record
     bool records_pending = true;
 
     const int tslot = warp / G, wsub = warp % G;
@@ -522,19 +560,23 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
         }
         // -- merged rows: a lane per row sums the entries into the row's virtual slot
         if (nslots > 0) {
-#pragma unroll 2
+            // the inline form is evaluated for every record (a longer row's record carries zero weights there), so
+            // that the loads of several records are in flight together; longer rows are patched afterwards
+#pragma unroll 4
             for (int vi = g0; vi < nslots; vi += GS) {
                 const uint4 r0 = s_vrec[2 * vi], r1 = s_vrec[2 * vi + 1];
-                float e;
-                if (r1.z <= uint32_t(kInline)) {           // unused entries carry weight 0 and position 0
-                    e = __uint_as_float(r0.z) * d[r0.x & 0xFFFFu];
-                    e = fmaf(__uint_as_float(r0.w), d[r0.x >> 16], e);
-                    e = fmaf(__uint_as_float(r1.x), d[r0.y & 0xFFFFu], e);
-                    e = fmaf(__uint_as_float(r1.y), d[r0.y >> 16], e);
-                } else {
-                    e = csr_row(rm, d, C, int(r0.x), int(r1.z));
-                }
+                float e = __uint_as_float(r0.z) * d[r0.x & 0xFFFFu];
+                e = fmaf(__uint_as_float(r0.w), d[r0.x >> 16], e);
+                e = fmaf(__uint_as_float(r1.x), d[r0.y & 0xFFFFu], e);
+                e = fmaf(__uint_as_float(r1.y), d[r0.y >> 16], e);
                 d[C + vi] = e;
+            }
+            if (nlong > 0) {                               // uniform over the grid; few rows
+                for (int vi = g0; vi < nslots; vi += GS) {
+                    const uint4 r1 = s_vrec[2 * vi + 1];
+                    if (r1.z > uint32_t(kInline))
+                        d[C + vi] = r1.w ? pair_row(s_lent, d, int(r1.x), int(r1.z)) : csr_row(rm, d, C, int(r1.x), int(r1.z));
+                }
             }
             token_sync<G>(barid);
         }
@@ -689,7 +731,8 @@ int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage&
     constexpr int C = NPL * 32 * G;
     auto kern = reassemble_quant_token<NPL, G, HAS_BETA, PACKED, MAXW>;
     const int row_words = C + slot_room;
-    const int64_t fixed = int64_t(HAS_BETA ? 12 : 8) * C + (MAXW / G) * 8 * G * 4 + int64_t(slot_room) * 32;   // records, exchange, slot records
+    const int64_t fixed = int64_t(HAS_BETA ? 12 : 8) * C + (MAXW / G) * 8 * G * 4 + int64_t(slot_room) * 32 +
+                          kLongCap * 8;   // records, exchange, slot records, entries of longer rows
     int tok_fit = int((kSmemBudget - fixed) / (int64_t(row_words) * 4));
     if (tok_fit > MAXW / G) tok_fit = MAXW / G;
     if (share_sm) {

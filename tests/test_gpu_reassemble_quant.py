@@ -71,11 +71,11 @@ def test_odd_channel_count_byte_codes():
     parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref, 6)
 
 
-@pytest.mark.parametrize("kind", ["long_rows", "slot_overflow", "identity"])
+@pytest.mark.parametrize("kind", ["long_rows", "many_long_rows", "slot_overflow", "identity"])
 @pytest.mark.parametrize("with_beta", [False, True])
 def test_handmade_maps_on_the_specialised_kernel(kind, with_beta):
     """Maps the builder would rarely produce, on a channel count the warp-per-token kernel serves:
-    rows with more entries than a slot record holds, more multi-entry rows than there are slots
+    rows with more entries than a slot record holds (few, and more than the image keeps), more multi-entry rows than there are slots
     (the launch then walks the CSR arrays), and the identity map."""
     import gpu_util as G
     rng = np.random.default_rng(11)
@@ -90,6 +90,10 @@ def test_handmade_maps_on_the_specialised_kernel(kind, with_beta):
     for c in range(C):
         if kind == "identity":
             rows.append([(c, 1.0)])
+        elif kind == "many_long_rows":                   # more long-row entries than the compiled image keeps
+            n = 6 if c % 3 == 0 else 1
+            srcs = [(c * 5 + 13 * e) % C for e in range(n)]
+            rows.append([(sj, 1.0 / n) for sj in srcs])
         elif kind == "long_rows":
             n = 1 + (c % 9 == 0) * (1 + c % 7)           # rows of 1 .. 7 entries
             srcs = [(c * 5 + 13 * e) % C for e in range(n)]
