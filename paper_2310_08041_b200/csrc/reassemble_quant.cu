@@ -35,6 +35,7 @@ namespace {
 constexpr int kSlotCap = 2048;                 // virtual slots an image can describe
 constexpr int kInline = 4;                     // entries held inside a slot record
 constexpr int kLongCap = 512;                  // entries of longer rows kept as (position, weight) pairs
+constexpr int kLongRows = 256;                 // longer rows listed by slot (more: the slot pass scans for them)
 constexpr int kMaxWarps = 16;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
@@ -94,6 +95,7 @@ __device__ __forceinline__ void prefetch_l2(const void* p) {
 //                            row whose entries fit lent; {0, 0, 0, 0}, {first CSR entry, 0, n, 0} otherwise (the
 //                            inline fields of such a record are harmless when evaluated: positions 0)
 //   lent uint2[kLongCap]     entries of the longer rows: {position, weight bits}
+//   lrow int[kLongRows]      slots of the longer rows, in no particular order
 //   head int[4]         [0] = slots handed out (more than kSlotCap: the map does not fit), [1] = entries handed
 //                       out in lent, [2] = rows longer than kInline
 struct WarpImage {
@@ -102,10 +104,11 @@ struct WarpImage {
     uint32_t *olo, *ohi;
     uint4* vrec;
     uint2* lent;
+    int* lrow;
     int* head;
 };
 __host__ __device__ inline size_t warp_image_bytes(int C) {
-    return size_t(C) * 14 + size_t(kSlotCap) * 32 + size_t(kLongCap) * 8 + 16;
+    return size_t(C) * 14 + size_t(kSlotCap) * 32 + size_t(kLongCap) * 8 + size_t(kLongRows) * 4 + 16;
 }
 __host__ __device__ inline WarpImage warp_image_at(void* base, int C) {
     WarpImage im;
@@ -119,7 +122,8 @@ __host__ __device__ inline WarpImage warp_image_at(void* base, int C) {
     im.ohi = im.olo + C / 2;
     im.vrec = reinterpret_cast<uint4*>(im.ohi + C / 2);
     im.lent = reinterpret_cast<uint2*>(im.vrec + 2 * size_t(kSlotCap));
-    im.head = reinterpret_cast<int*>(im.lent + kLongCap);
+    im.lrow = reinterpret_cast<int*>(im.lent + kLongCap);
+    im.head = im.lrow + kLongRows;
     return im;
 }
 
@@ -166,7 +170,8 @@ compile_map_warp_kernel(int C, const float* __restrict__ gamma, const float* __r
                     im.vrec[2 * vi] = make_uint4(0u, 0u, 0u, 0u);
                     im.vrec[2 * vi + 1] = make_uint4(uint32_t(j0), 0u, uint32_t(n), 0u);
                 }
-                atomicAdd(im.head + 2, 1);                // number of longer rows
+                const int li = atomicAdd(im.head + 2, 1);   // number of longer rows
+                if (li < kLongRows) im.lrow[li] = vi;
             }
             pos = uint32_t(C + vi);
             w = 1.0f;
@@ -467,7 +472,8 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
     float* s_ex = reinterpret_cast<float*>(s_offB + C / 2);             // [MAXW / G][8 G] exchange words per token slot
     uint4* s_vrec = reinterpret_cast<uint4*>(s_ex + (MAXW / G) * 8 * G);   // [row_words - C][2] slot records
     uint2* s_lent = reinterpret_cast<uint2*>(s_vrec + 2 * size_t(row_words - C));   // [kLongCap] entries of longer rows
-    float* rows = reinterpret_cast<float*>(s_lent + kLongCap);
+    int* s_lrow = reinterpret_cast<int*>(s_lent + kLongCap);                    // [kLongRows] their slots
+    float* rows = reinterpret_cast<float*>(s_lrow + kLongRows);
 
     const int lane = threadIdx.x & 31;
     const int warp = __shfl_sync(0xffffffffu, int(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
@@ -487,6 +493,8 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
         for (int i = threadIdx.x; i < 2 * (row_words - C); i += blockDim.x) cp_async16(s_vrec + i, im.vrec + i);
         for (int i = threadIdx.x; i < kLongCap / 2; i += blockDim.x)
             cp_async16(reinterpret_cast<uint4*>(s_lent) + i, reinterpret_cast<const uint4*>(im.lent) + i);
+        for (int i = threadIdx.x; i < kLongRows / 4; i += blockDim.x)
+            cp_async16(reinterpret_cast<uint4*>(s_lrow) + i, reinterpret_cast<const uint4*>(im.lrow) + i);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
     const int slots_total = __ldg(im.head);
@@ -572,7 +580,9 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
                 d[C + vi] = e;
             }
             if (nlong > 0) {                               // uniform over the grid; few rows
-                for (int vi = g0; vi < nslots; vi += GS) {
+                const bool listed = nlong <= kLongRows;
+                for (int k = g0; k < (listed ? nlong : nslots); k += GS) {
+                    const int vi = listed ? s_lrow[k] : k;
                     const uint4 r1 = s_vrec[2 * vi + 1];
                     if (r1.z > uint32_t(kInline))
                         d[C + vi] = r1.w ? pair_row(s_lent, d, int(r1.x), int(r1.z)) : csr_row(rm, d, C, int(r1.x), int(r1.z));
@@ -732,7 +742,7 @@ int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage&
     auto kern = reassemble_quant_token<NPL, G, HAS_BETA, PACKED, MAXW>;
     const int row_words = C + slot_room;
     const int64_t fixed = int64_t(HAS_BETA ? 12 : 8) * C + (MAXW / G) * 8 * G * 4 + int64_t(slot_room) * 32 +
-                          kLongCap * 8;   // records, exchange, slot records, entries of longer rows
+                          kLongCap * 8 + kLongRows * 4;   // records, exchange, slot records, longer rows
     int tok_fit = int((kSmemBudget - fixed) / (int64_t(row_words) * 4));
     if (tok_fit > MAXW / G) tok_fit = MAXW / G;
     if (share_sm) {
