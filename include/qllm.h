@@ -291,7 +291,9 @@ int qllm_layer_forward(qllm_layer_t* layer, const void* x, int64_t M, void* out,
 int qllm_layer_reassemble_quant(qllm_layer_t* layer, const void* x, int64_t M, void* stream);
 int qllm_layer_qgemm(qllm_layer_t* layer, int64_t M, void* out, void* stream);
 /* x, out: HOST (pinned memory makes the copies asynchronous).  Copies x to the device, runs the
- * path, copies out back and waits for the stream. */
+ * path, copies out back and waits until all of it is done.  Calls of 2048 tokens or more are cut into four
+ * chunks of token rows whose copy in, kernels and copy out overlap on two internal copy streams (the host link
+ * carries both directions at once); results are those of qllm_layer_forward. */
 int qllm_layer_forward_host(qllm_layer_t* layer, const void* x_host, int64_t M, void* out_host,
                             void* stream);
 /* Borrowed DEVICE pointers of the layer's quantized-activation workspace of the last forward.

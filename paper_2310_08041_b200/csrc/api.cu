@@ -171,6 +171,10 @@ struct qllm_layer {
     // pre-GEMM call starts it on a side stream; the GEMM call joins it.
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // host-buffer calls of many tokens run in chunks so that the copy in, the kernels and the copy out overlap
+    static constexpr int kHostChunks = 4;
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
     const uint8_t* w_ready = nullptr;            // expanded weights in flight / ready for the next GEMM call
     int64_t w_ready_M = -1;
     // 4-bit activations of a call that will take the byte-lane GEMM are written one code per byte by the
@@ -318,6 +322,11 @@ void qllm_layer_destroy(qllm_layer_t* L) {
     if (L->side) { cudaStreamSynchronize(L->side); cudaStreamDestroy(L->side); }
     if (L->ev_fork) cudaEventDestroy(L->ev_fork);
     if (L->ev_join) cudaEventDestroy(L->ev_join);
+    if (L->h2d) { cudaStreamSynchronize(L->h2d); cudaStreamDestroy(L->h2d); }
+    if (L->d2h) { cudaStreamSynchronize(L->d2h); cudaStreamDestroy(L->d2h); }
+    if (L->ev_start) cudaEventDestroy(L->ev_start);
+    for (cudaEvent_t e : L->ev_in) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : L->ev_done) if (e) cudaEventDestroy(e);
     for (void* p : L->owned) cudaFree(p);
     delete L;
 }
@@ -376,11 +385,60 @@ int qllm_layer_forward_host(qllm_layer_t* L, const void* x_host, int64_t M, void
     if (M == 0) return QLLM_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t xb = L->x_dtype == QLLM_F32 ? 4 : 2, ob = L->out_dtype == QLLM_F32 ? 4 : 2;
-    QLLM_CUDA_TRY(cudaMemcpyAsync(L->x_dev, x_host, size_t(M) * L->C * xb, cudaMemcpyHostToDevice, st));
-    int rc = qllm_layer_forward(L, L->x_dev, M, L->out_dev, stream);
+    constexpr int NC = qllm_layer::kHostChunks;
+    const int64_t rows = ((M + NC - 1) / NC + 127) / 128 * 128;      // tokens per chunk
+    if (rows < kExpandMinM || rows >= M) {
+        // few tokens: one copy in, the path, one copy out
+        QLLM_CUDA_TRY(cudaMemcpyAsync(L->x_dev, x_host, size_t(M) * L->C * xb, cudaMemcpyHostToDevice, st));
+        int rc = qllm_layer_forward(L, L->x_dev, M, L->out_dev, stream);
+        if (rc != QLLM_OK) return rc;
+        QLLM_CUDA_TRY(cudaMemcpyAsync(out_host, L->out_dev, size_t(M) * L->N * ob, cudaMemcpyDeviceToHost, st));
+        QLLM_CUDA_TRY(cudaStreamSynchronize(st));
+        return QLLM_OK;
+    }
+    // Many tokens: the copies dominate (x in, out back over the host link), so the call is cut into chunks of
+    // token rows: chunk k + 1 is copied in and chunk k - 1 copied out on two copy streams while chunk k runs.
+    if (!L->h2d) {
+        if (cudaStreamCreateWithFlags(&L->h2d, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&L->d2h, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&L->ev_start, cudaEventDisableTiming) != cudaSuccess)
+            return cuda_fail(cudaGetLastError());
+        for (int k = 0; k < NC; ++k)
+            if (cudaEventCreateWithFlags(&L->ev_in[k], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&L->ev_done[k], cudaEventDisableTiming) != cudaSuccess)
+                return cuda_fail(cudaGetLastError());
+    }
+    const char* xh = static_cast<const char*>(x_host);
+    char* oh = static_cast<char*>(out_host);
+    char* xd = static_cast<char*>(L->x_dev);
+    char* od = static_cast<char*>(L->out_dev);
+    QLLM_CUDA_TRY(cudaEventRecord(L->ev_start, st));                 // earlier work on the caller's stream first
+    QLLM_CUDA_TRY(cudaStreamWaitEvent(L->h2d, L->ev_start, 0));
+    int nk = 0;
+    for (int64_t m0 = 0; m0 < M; m0 += rows, ++nk) {
+        const int64_t mk = std::min<int64_t>(rows, M - m0);
+        QLLM_CUDA_TRY(cudaMemcpyAsync(xd + size_t(m0) * L->C * xb, xh + size_t(m0) * L->C * xb, size_t(mk) * L->C * xb,
+                                      cudaMemcpyHostToDevice, L->h2d));
+        QLLM_CUDA_TRY(cudaEventRecord(L->ev_in[nk], L->h2d));
+    }
+    int rc = QLLM_OK;
+    nk = 0;
+    for (int64_t m0 = 0; m0 < M && rc == QLLM_OK; m0 += rows, ++nk) {
+        const int64_t mk = std::min<int64_t>(rows, M - m0);
+        QLLM_CUDA_TRY(cudaStreamWaitEvent(st, L->ev_in[nk], 0));
+        rc = qllm_layer_forward(L, xd + size_t(m0) * L->C * xb, mk, od + size_t(m0) * L->N * ob, stream);
+        if (rc != QLLM_OK) break;
+        QLLM_CUDA_TRY(cudaEventRecord(L->ev_done[nk], st));
+        QLLM_CUDA_TRY(cudaStreamWaitEvent(L->d2h, L->ev_done[nk], 0));
+        QLLM_CUDA_TRY(cudaMemcpyAsync(oh + size_t(m0) * L->N * ob, od + size_t(m0) * L->N * ob, size_t(mk) * L->N * ob,
+                                      cudaMemcpyDeviceToHost, L->d2h));
+    }
+    // nothing of this call may be in flight when it returns, whatever happened
+    const cudaError_t e1 = cudaStreamSynchronize(L->h2d), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(L->d2h);
     if (rc != QLLM_OK) return rc;
-    QLLM_CUDA_TRY(cudaMemcpyAsync(out_host, L->out_dev, size_t(M) * L->N * ob, cudaMemcpyDeviceToHost, st));
-    QLLM_CUDA_TRY(cudaStreamSynchronize(st));
+    if (e1 != cudaSuccess) return cuda_fail(e1);
+    if (e2 != cudaSuccess) return cuda_fail(e2);
+    if (e3 != cudaSuccess) return cuda_fail(e3);
     return QLLM_OK;
 }
 

@@ -122,4 +122,9 @@ def test_layer_full_size_two_halves_sampled(name):
                                     L["w_scale"][n:n + 1], L["w_zero"][n:n + 1], L["w_colsum"][n:n + 1])[0, 0]
                     for a, m, n in zip(acc, ms, ns)])
     parity.check_output(G.bf16_bits(out.cpu())[ms, ns], ref, "bf16")
+    # the host-buffer entry point (chunked and overlapped at this size) returns the same bytes
+    xh = torch.from_numpy(x.view(np.int16)).pin_memory()
+    oh = torch.zeros((M, N), dtype=torch.bfloat16).pin_memory()
+    layer.forward_host(xh, oh, M)
+    assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
     layer.destroy()
