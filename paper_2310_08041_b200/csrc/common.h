@@ -75,8 +75,8 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
                             const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
                             float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes = false,
                             int slots_known = -1, bool share_sm = false);
-// Multi-entry rows of a compiled image (waits for the stream); passing it to the launcher as slots_known
-// sizes the kernel's shared-memory rows exactly instead of for the largest image.  share_sm: another kernel
+// Counts of the multi-entry rows of a compiled image, packed into one int (waits for the stream); passing it to
+// the launcher as slots_known sizes the kernel's shared memory exactly instead of for the largest image.  share_sm: another kernel
 // of the caller runs beside this one; leave part of each SM's registers to it.
 int reassemble_map_slots(int C, const void* image, cudaStream_t st, int* slots);
 int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C, const float* gamma,

@@ -88,27 +88,33 @@ __device__ __forceinline__ void prefetch_l2(const void* p) {
 //   idx  uint16[C]      word position in the row of the channel's (first or only) source, or C + slot
 //   wlo  float[C/8][4]  weights of channels 8g .. 8g+3        whi: channels 8g+4 .. 8g+7
 //   blo, bhi            bias terms in the same layout (zero without beta)
-//   olo, ohi uint32[C/8][4]  the positions again as byte offsets (4 * idx), in the weights' layout
-//   vrec uint4[kSlotCap][2]  slot s: {pos0 | pos1 << 16, pos2 | pos3 << 16, w0, w1}, {w2, w3, n, 0}
-//                            for n <= kInline entries; {first CSR entry, -, -, -}, {-, -, n, 0} otherwise
-//                            for n <= kInline entries; {0, 0, 0, 0}, {first entry in lent, 0, n, 1} for a longer
-//                            row whose entries fit lent; {0, 0, 0, 0}, {first CSR entry, 0, n, 0} otherwise (the
-//                            inline fields of such a record are harmless when evaluated: positions 0)
-//   lent uint2[kLongCap]     entries of the longer rows: {position, weight bits}
-//   lrow int[kLongRows]      slots of the longer rows, in no particular order
-//   head int[4]         [0] = slots handed out (more than kSlotCap: the map does not fit), [1] = entries handed
-//                       out in lent, [2] = rows longer than kInline
+//   Virtual slots, rows of two entries first (slots 0 .. n2-1), rows of three and more after them
+//   (slots n2 .. n2+n34-1), each field an array of its own so that a warp reads them without bank conflicts:
+//   p01 uint32[kSlotCap], w0, w1 float[kSlotCap]     pos0 | pos1 << 16 and the two weights, every slot
+//   p23 uint32[kOtherCap], w2, w3 float[kOtherCap]   entries 2 and 3 of slot n2 + t (weight 0 where absent)
+//   A row longer than kInline entries has zero weights in those fields and is listed in
+//   lmeta int4[kLongRows]    {slot, first, n, kind}: kind 1 = entries lent[first .. first+n), kind 0 = CSR entries
+//   lent uint2[kLongCap]     {position, weight bits}
+//   head int[8]         [0], [3] = pairs / other rows given a slot so far (assign kernel), [1] = entries handed out in
+//                       lent, [2] = rows longer than kInline listed so far, [4] = n2, [5] = n34, [6] = rows longer
+//                       than kInline (count kernel)
+// The slots serve a launch when n2 + n34 <= the row's slot room, n34 <= the room for p23/w2/w3 and all longer
+// rows are listed; otherwise the launch walks the CSR arrays.
+constexpr int kOtherCap = 1024;
 struct WarpImage {
     uint16_t* idx;
     float *wlo, *whi, *blo, *bhi;
-    uint32_t *olo, *ohi;
-    uint4* vrec;
+    uint32_t* p01;
+    float *w0, *w1;
+    uint32_t* p23;
+    float *w2, *w3;
+    int4* lmeta;
     uint2* lent;
-    int* lrow;
     int* head;
 };
 __host__ __device__ inline size_t warp_image_bytes(int C) {
-    return size_t(C) * 14 + size_t(kSlotCap) * 32 + size_t(kLongCap) * 8 + size_t(kLongRows) * 4 + 16;
+    return size_t(C) * 10 + size_t(kSlotCap) * 12 + size_t(kOtherCap) * 12 + size_t(kLongRows) * 16 +
+           size_t(kLongCap) * 8 + 32;
 }
 __host__ __device__ inline WarpImage warp_image_at(void* base, int C) {
     WarpImage im;
@@ -118,22 +124,42 @@ __host__ __device__ inline WarpImage warp_image_at(void* base, int C) {
     im.whi = im.wlo + C / 2;
     im.blo = im.whi + C / 2;
     im.bhi = im.blo + C / 2;
-    im.olo = reinterpret_cast<uint32_t*>(im.bhi + C / 2);
-    im.ohi = im.olo + C / 2;
-    im.vrec = reinterpret_cast<uint4*>(im.ohi + C / 2);
-    im.lent = reinterpret_cast<uint2*>(im.vrec + 2 * size_t(kSlotCap));
-    im.lrow = reinterpret_cast<int*>(im.lent + kLongCap);
-    im.head = im.lrow + kLongRows;
+    im.p01 = reinterpret_cast<uint32_t*>(im.bhi + C / 2);
+    im.w0 = reinterpret_cast<float*>(im.p01 + kSlotCap);
+    im.w1 = im.w0 + kSlotCap;
+    im.p23 = reinterpret_cast<uint32_t*>(im.w1 + kSlotCap);
+    im.w2 = reinterpret_cast<float*>(im.p23 + kOtherCap);
+    im.w3 = im.w2 + kOtherCap;
+    im.lmeta = reinterpret_cast<int4*>(im.w3 + kOtherCap);
+    im.lent = reinterpret_cast<uint2*>(im.lmeta + kLongRows);
+    im.head = reinterpret_cast<int*>(im.lent + kLongCap);
     return im;
 }
 
-// One thread per output channel.  im.head[0] must be zero at launch.
+__device__ __forceinline__ bool slots_fit(const int* head, int slot_room, int other_room) {
+    return head[4] + head[5] <= slot_room && head[5] <= other_room && head[6] <= kLongRows;
+}
+
+// Pass 1: how many rows have two entries, how many more.  head must be zero at launch.
+__global__ void __launch_bounds__(256)
+count_rows_kernel(int C, const int32_t* __restrict__ ptr, WarpImage im) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    const int n = __ldg(ptr + c + 1) - __ldg(ptr + c);
+    if (n == 2) atomicAdd(im.head + 4, 1);
+    else if (n > 2) atomicAdd(im.head + 5, 1);
+    if (n > kInline) atomicAdd(im.head + 6, 1);
+}
+
+// Pass 2: one thread per output channel writes its record and, for a multi-entry row, its slot.
 __global__ void __launch_bounds__(256)
 compile_map_warp_kernel(int C, const float* __restrict__ gamma, const float* __restrict__ beta,
                         const int32_t* __restrict__ ptr, const int32_t* __restrict__ src,
                         const float* __restrict__ coef, WarpImage im) {
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= C) return;
+    const int n2 = im.head[4], n34 = im.head[5];
+    const bool fits = slots_fit(im.head, kSlotCap, kOtherCap);
     const int j0 = __ldg(ptr + c), n = __ldg(ptr + c + 1) - j0;
     const int s0 = __ldg(src + j0);
     const float c0 = __ldg(coef + j0);
@@ -143,37 +169,44 @@ compile_map_warp_kernel(int C, const float* __restrict__ gamma, const float* __r
     if (n > 1) {                                          // merged row
         if (beta)
             for (int j = j0 + 1; j < j0 + n; ++j) b = fmaf(__ldg(coef + j), __ldg(beta + __ldg(src + j)), b);
-        const int vi = atomicAdd(im.head, 1);
-        if (vi < kSlotCap) {
-            if (n <= kInline) {
-                uint32_t o[kInline] = {0, 0, 0, 0};
-                float ww[kInline] = {0.f, 0.f, 0.f, 0.f};
+        if (fits) {
+            uint32_t o[kInline] = {0, 0, 0, 0};
+            float ww[kInline] = {0.f, 0.f, 0.f, 0.f};
+            if (n <= kInline)
                 for (int e = 0; e < n; ++e) {
                     const int sj = __ldg(src + j0 + e);
                     o[e] = uint32_t(dplane(sj, C));
                     ww[e] = __ldg(coef + j0 + e) * __ldg(gamma + sj);
                 }
-                im.vrec[2 * vi] = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), __float_as_uint(ww[0]),
-                                             __float_as_uint(ww[1]));
-                im.vrec[2 * vi + 1] = make_uint4(__float_as_uint(ww[2]), __float_as_uint(ww[3]), uint32_t(n), 0u);
+            int slot;
+            if (n == 2) {
+                slot = atomicAdd(im.head, 1);
             } else {
-                const int first = atomicAdd(im.head + 1, n);
+                const int t = atomicAdd(im.head + 3, 1);
+                slot = n2 + t;
+                im.p23[t] = o[2] | (o[3] << 16);
+                im.w2[t] = ww[2];
+                im.w3[t] = ww[3];
+            }
+            im.p01[slot] = o[0] | (o[1] << 16);
+            im.w0[slot] = ww[0];
+            im.w1[slot] = ww[1];
+            if (n > kInline) {
+                int first = atomicAdd(im.head + 1, n), kind = 1;
                 if (first + n <= kLongCap) {              // entries as (position, weight) pairs for shared memory
                     for (int e = 0; e < n; ++e) {
                         const int sj = __ldg(src + j0 + e);
                         im.lent[first + e] = make_uint2(uint32_t(dplane(sj, C)),
                                                         __float_as_uint(__ldg(coef + j0 + e) * __ldg(gamma + sj)));
                     }
-                    im.vrec[2 * vi] = make_uint4(0u, 0u, 0u, 0u);
-                    im.vrec[2 * vi + 1] = make_uint4(uint32_t(first), 0u, uint32_t(n), 1u);
                 } else {                                  // walks the CSR arrays at run time
-                    im.vrec[2 * vi] = make_uint4(0u, 0u, 0u, 0u);
-                    im.vrec[2 * vi + 1] = make_uint4(uint32_t(j0), 0u, uint32_t(n), 0u);
+                    first = j0;
+                    kind = 0;
                 }
-                const int li = atomicAdd(im.head + 2, 1);   // number of longer rows
-                if (li < kLongRows) im.lrow[li] = vi;
+                const int li = atomicAdd(im.head + 2, 1);
+                if (li < kLongRows) im.lmeta[li] = make_int4(slot, first, n, kind);
             }
-            pos = uint32_t(C + vi);
+            pos = uint32_t(C + slot);
             w = 1.0f;
         }
     }
@@ -181,7 +214,6 @@ compile_map_warp_kernel(int C, const float* __restrict__ gamma, const float* __r
     const int g = c >> 3, j = c & 7;
     (j < 4 ? im.wlo : im.whi)[4 * g + (j & 3)] = w;
     (j < 4 ? im.blo : im.bhi)[4 * g + (j & 3)] = b;
-    (j < 4 ? im.olo : im.ohi)[4 * g + (j & 3)] = pos * 4u;
 }
 
 // 8 consecutive channels of a row as floats
@@ -278,10 +310,10 @@ reassemble_quant_warp(const XT* __restrict__ x, int64_t M, int C, float eps, int
         const int n16 = (HAS_BETA ? 10 : 6) * C / 16;
         for (int i = threadIdx.x; i < n16; i += blockDim.x) s4[i] = __ldg(g4 + i);
     }
-    const int slots_total = __ldg(im.head);
-    const int slot_room = row_words - C;
-    const bool slow = slots_total > slot_room;             // uniform over the grid
-    const int nslots = slow ? 0 : slots_total;
+    const bool slow = !slots_fit(im.head, row_words - C, kOtherCap);   // uniform over the grid
+    const int n2 = slow ? 0 : __ldg(im.head + 4);
+    const int nslots = slow ? 0 : n2 + __ldg(im.head + 5);
+    const int nlong = slow ? 0 : __ldg(im.head + 6);
     __syncthreads();
 
     float* d = rows + size_t(warp) * row_words;
@@ -325,21 +357,19 @@ reassemble_quant_warp(const XT* __restrict__ x, int64_t M, int C, float eps, int
         __syncwarp();
         // -- merged rows: a lane per row sums the entries into the row's virtual slot
         for (int vi = lane; vi < nslots; vi += 32) {
-            const uint4 r0 = __ldg(im.vrec + 2 * vi), r1 = __ldg(im.vrec + 2 * vi + 1);
-            float e;
-            if (r1.z <= uint32_t(kInline)) {
-                e = __uint_as_float(r0.z) * d[r0.x & 0xFFFFu];
-                e = fmaf(__uint_as_float(r0.w), d[r0.x >> 16], e);
-                if (r1.z > 2u) {
-                    e = fmaf(__uint_as_float(r1.x), d[r0.y & 0xFFFFu], e);
-                    if (r1.z > 3u) e = fmaf(__uint_as_float(r1.y), d[r0.y >> 16], e);
-                }
-            } else if (r1.w) {
-                e = pair_row(im.lent, d, int(r1.x), int(r1.z));
-            } else {
-                e = csr_row(rm, d, C, int(r1.x), int(r1.z));
+            const uint32_t p = __ldg(im.p01 + vi);
+            float e = __ldg(im.w0 + vi) * d[p & 0xFFFFu];
+            e = fmaf(__ldg(im.w1 + vi), d[p >> 16], e);
+            if (vi >= n2) {
+                const uint32_t q = __ldg(im.p23 + vi - n2);
+                e = fmaf(__ldg(im.w2 + vi - n2), d[q & 0xFFFFu], e);
+                e = fmaf(__ldg(im.w3 + vi - n2), d[q >> 16], e);
             }
             d[C + vi] = e;
+        }
+        for (int k = lane; k < nlong; k += 32) {               // the few rows longer than a record
+            const int4 lm = __ldg(im.lmeta + k);
+            d[C + lm.x] = lm.w ? pair_row(im.lent, d, lm.y, lm.z) : csr_row(rm, d, C, lm.y, lm.z);
         }
         __syncwarp();
         // -- row range of x' (first gather pass)
@@ -433,7 +463,8 @@ reassemble_quant_warp(const XT* __restrict__ x, int64_t M, int C, float eps, int
 // a lane owns NPL = C / (32 G) channels, 8 consecutive ones per step.  The whole row is loaded
 // with all its 16-byte loads in flight, converted once, and the reassembled values x' stay in
 // registers between the range pass and the quantize pass, so each channel is gathered once.
-// Records are kept as 32-bit byte offsets so that a gather is one shared load at [offset + row].
+// Positions stay 16-bit and slot records are split by field (and by row length) in shared memory: what limits
+// the kernel is the number of shared-memory wavefronts per token and the tokens that fit beside the records.
 template <int G>
 __device__ __forceinline__ void token_sync(int barid) {
     if (G == 1) __syncwarp();
@@ -456,7 +487,8 @@ __device__ __forceinline__ float token_sum(float v, float* ex, int& par, int wsu
 template <int NPL, int G, bool HAS_BETA, bool PACKED, int MAXW>
 __global__ void __launch_bounds__(32 * MAXW, 1)
 reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps, int bits, WarpImage im,
-                       int row_words, int TOK /* tokens in flight per CTA */, RawMap rm, uint8_t* __restrict__ codes, float* __restrict__ a_scale,
+                       int row_words, int other_room, int TOK /* tokens in flight per CTA */, RawMap rm,
+                       uint8_t* __restrict__ codes, float* __restrict__ a_scale,
                        float* __restrict__ a_zero, int32_t* __restrict__ a_rowsum) {
     constexpr int C = NPL * 32 * G;
     constexpr int NIT = NPL / 8;                           // steps of 8 channels per lane
@@ -467,13 +499,18 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
     float* s_wB = s_wA + C / 2;                            //                      channels 8g+4..8g+7
     float* s_bA = s_wB + C / 2;                            // bias arrays only with beta
     float* s_bB = s_bA + C / 2;
-    uint32_t* s_offA = reinterpret_cast<uint32_t*>(HAS_BETA ? s_bB + C / 2 : s_bA);   // byte offsets, same layout
-    uint32_t* s_offB = s_offA + C / 2;
-    float* s_ex = reinterpret_cast<float*>(s_offB + C / 2);             // [MAXW / G][8 G] exchange words per token slot
-    uint4* s_vrec = reinterpret_cast<uint4*>(s_ex + (MAXW / G) * 8 * G);   // [row_words - C][2] slot records
-    uint2* s_lent = reinterpret_cast<uint2*>(s_vrec + 2 * size_t(row_words - C));   // [kLongCap] entries of longer rows
-    int* s_lrow = reinterpret_cast<int*>(s_lent + kLongCap);                    // [kLongRows] their slots
-    float* rows = reinterpret_cast<float*>(s_lrow + kLongRows);
+    uint16_t* s_idx = reinterpret_cast<uint16_t*>(HAS_BETA ? s_bB + C / 2 : s_bA);     // [C] word positions
+    float* s_ex = reinterpret_cast<float*>(s_idx + C);                  // [MAXW / G][8 G] exchange words per token slot
+    const int slot_room = row_words - C;
+    uint32_t* s_p01 = reinterpret_cast<uint32_t*>(s_ex + (MAXW / G) * 8 * G);   // slot records, field by field
+    float* s_w0 = reinterpret_cast<float*>(s_p01 + slot_room);
+    float* s_w1 = s_w0 + slot_room;
+    uint32_t* s_p23 = reinterpret_cast<uint32_t*>(s_w1 + slot_room);
+    float* s_w2 = reinterpret_cast<float*>(s_p23 + other_room);
+    float* s_w3 = s_w2 + other_room;
+    int4* s_lmeta = reinterpret_cast<int4*>(s_w3 + other_room);                 // [kLongRows] rows longer than a record
+    uint2* s_lent = reinterpret_cast<uint2*>(s_lmeta + kLongRows);              // [kLongCap] their entries
+    float* rows = reinterpret_cast<float*>(s_lent + kLongCap);
 
     const int lane = threadIdx.x & 31;
     const int warp = __shfl_sync(0xffffffffu, int(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
@@ -488,19 +525,25 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
         const uint4* gw = reinterpret_cast<const uint4*>(im.wlo);       // wlo | whi | blo | bhi back to back
         const int nw16 = (HAS_BETA ? 8 : 4) * C / 16;
         for (int i = threadIdx.x; i < nw16; i += blockDim.x) cp_async16(reinterpret_cast<uint4*>(s_wA) + i, gw + i);
-        const uint4* go = reinterpret_cast<const uint4*>(im.olo);       // olo | ohi back to back
-        for (int i = threadIdx.x; i < 4 * C / 16; i += blockDim.x) cp_async16(reinterpret_cast<uint4*>(s_offA) + i, go + i);
-        for (int i = threadIdx.x; i < 2 * (row_words - C); i += blockDim.x) cp_async16(s_vrec + i, im.vrec + i);
-        for (int i = threadIdx.x; i < kLongCap / 2; i += blockDim.x)
-            cp_async16(reinterpret_cast<uint4*>(s_lent) + i, reinterpret_cast<const uint4*>(im.lent) + i);
-        for (int i = threadIdx.x; i < kLongRows / 4; i += blockDim.x)
-            cp_async16(reinterpret_cast<uint4*>(s_lrow) + i, reinterpret_cast<const uint4*>(im.lrow) + i);
+        auto copy16 = [&](void* dst, const void* src, int n16) {
+            for (int i = threadIdx.x; i < n16; i += blockDim.x)
+                cp_async16(static_cast<uint4*>(dst) + i, static_cast<const uint4*>(src) + i);
+        };
+        copy16(s_idx, im.idx, 2 * C / 16);
+        copy16(s_p01, im.p01, slot_room / 4);
+        copy16(s_w0, im.w0, slot_room / 4);
+        copy16(s_w1, im.w1, slot_room / 4);
+        copy16(s_p23, im.p23, other_room / 4);
+        copy16(s_w2, im.w2, other_room / 4);
+        copy16(s_w3, im.w3, other_room / 4);
+        copy16(s_lmeta, im.lmeta, kLongRows);
+        copy16(s_lent, im.lent, kLongCap / 2);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    const int slots_total = __ldg(im.head);
-    const bool slow = slots_total > row_words - C;         // uniform over the grid: walk the CSR arrays
-    const int nslots = slow ? 0 : slots_total;
-    const int nlong = __ldg(im.head + 2);                  // rows longer than a slot record
+    const bool slow = !slots_fit(im.head, slot_room, other_room);   // uniform over the grid: walk the CSR arrays
+    const int n2 = slow ? 0 : __ldg(im.head + 4);          // slots of two-entry rows come first
+    const int nslots = slow ? 0 : n2 + __ldg(im.head + 5);
+    const int nlong = slow ? 0 : __ldg(im.head + 6);       // rows longer than a slot record
     bool records_pending = true;
 
     const int tslot = warp / G, wsub = warp % G;
@@ -513,7 +556,6 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
     float* d = rows + size_t(tslot) * row_words;
     float* ex = s_ex + tslot * 8 * G;
     float* exr = ex + 2 * G;                               // range exchange: [2][G][2]
-    const char* dbytes = reinterpret_cast<const char*>(d);
     const int g0 = wsub * 32 + lane;                       // this lane's group in step 0
     const float invC = 1.0f / float(C);
     const float qmax = float((1 << bits) - 1);
@@ -568,25 +610,23 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
         }
         // -- merged rows: a lane per row sums the entries into the row's virtual slot
         if (nslots > 0) {
-            // the inline form is evaluated for every record (a longer row's record carries zero weights there), so
-            // that the loads of several records are in flight together; longer rows are patched afterwards
+            // two-entry rows first, then the rows with entries 2 and 3 (only the warp step that straddles n2 diverges);
+            // a longer row's record carries zero weights and is patched afterwards
 #pragma unroll 4
             for (int vi = g0; vi < nslots; vi += GS) {
-                const uint4 r0 = s_vrec[2 * vi], r1 = s_vrec[2 * vi + 1];
-                float e = __uint_as_float(r0.z) * d[r0.x & 0xFFFFu];
-                e = fmaf(__uint_as_float(r0.w), d[r0.x >> 16], e);
-                e = fmaf(__uint_as_float(r1.x), d[r0.y & 0xFFFFu], e);
-                e = fmaf(__uint_as_float(r1.y), d[r0.y >> 16], e);
+                const uint32_t p = s_p01[vi];
+                float e = s_w0[vi] * d[p & 0xFFFFu];
+                e = fmaf(s_w1[vi], d[p >> 16], e);
+                if (vi >= n2) {
+                    const uint32_t q = s_p23[vi - n2];
+                    e = fmaf(s_w2[vi - n2], d[q & 0xFFFFu], e);
+                    e = fmaf(s_w3[vi - n2], d[q >> 16], e);
+                }
                 d[C + vi] = e;
             }
-            if (nlong > 0) {                               // uniform over the grid; few rows
-                const bool listed = nlong <= kLongRows;
-                for (int k = g0; k < (listed ? nlong : nslots); k += GS) {
-                    const int vi = listed ? s_lrow[k] : k;
-                    const uint4 r1 = s_vrec[2 * vi + 1];
-                    if (r1.z > uint32_t(kInline))
-                        d[C + vi] = r1.w ? pair_row(s_lent, d, int(r1.x), int(r1.z)) : csr_row(rm, d, C, int(r1.x), int(r1.z));
-                }
+            for (int k = g0; k < nlong; k += GS) {         // few rows
+                const int4 lm = s_lmeta[k];
+                d[C + lm.x] = lm.w ? pair_row(s_lent, d, lm.y, lm.z) : csr_row(rm, d, C, lm.y, lm.z);
             }
             token_sync<G>(barid);
         }
@@ -596,21 +636,17 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
 #pragma unroll
         for (int i = 0; i < NIT; ++i) {
             const int g = g0 + i * GS;
-            const uint4 oa = reinterpret_cast<const uint4*>(s_offA)[g], ob = reinterpret_cast<const uint4*>(s_offB)[g];
+            const uint4 iw = reinterpret_cast<const uint4*>(s_idx)[g];     // 8 word positions
             const float4 wa = reinterpret_cast<const float4*>(s_wA)[g], wb = reinterpret_cast<const float4*>(s_wB)[g];
             float* u = v + 8 * i;
             if (slow) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) u[j] = csr_channel(rm, d, C, 8 * g + j);
             } else {
-            u[0] = wa.x * *reinterpret_cast<const float*>(dbytes + oa.x);
-            u[1] = wa.y * *reinterpret_cast<const float*>(dbytes + oa.y);
-            u[2] = wa.z * *reinterpret_cast<const float*>(dbytes + oa.z);
-            u[3] = wa.w * *reinterpret_cast<const float*>(dbytes + oa.w);
-            u[4] = wb.x * *reinterpret_cast<const float*>(dbytes + ob.x);
-            u[5] = wb.y * *reinterpret_cast<const float*>(dbytes + ob.y);
-            u[6] = wb.z * *reinterpret_cast<const float*>(dbytes + ob.z);
-            u[7] = wb.w * *reinterpret_cast<const float*>(dbytes + ob.w);
+            u[0] = wa.x * d[iw.x & 0xFFFFu]; u[1] = wa.y * d[iw.x >> 16];
+            u[2] = wa.z * d[iw.y & 0xFFFFu]; u[3] = wa.w * d[iw.y >> 16];
+            u[4] = wb.x * d[iw.z & 0xFFFFu]; u[5] = wb.y * d[iw.z >> 16];
+            u[6] = wb.z * d[iw.w & 0xFFFFu]; u[7] = wb.w * d[iw.w >> 16];
             }
             if (HAS_BETA) {
                 const float4 ba = reinterpret_cast<const float4*>(s_bA)[g], bb = reinterpret_cast<const float4*>(s_bB)[g];
@@ -736,13 +772,15 @@ int launch_warp(const void* x, int64_t M, int C, float eps, int bits, const Warp
 
 
 template <int NPL, int G, bool HAS_BETA, bool PACKED, int MAXW>
-int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage& im, int slot_room, const RawMap& rm,
+int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage& im, int slot_room, int other_room,
+                 const RawMap& rm,
                  uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool share_sm) {
     constexpr int C = NPL * 32 * G;
     auto kern = reassemble_quant_token<NPL, G, HAS_BETA, PACKED, MAXW>;
     const int row_words = C + slot_room;
-    const int64_t fixed = int64_t(HAS_BETA ? 12 : 8) * C + (MAXW / G) * 8 * G * 4 + int64_t(slot_room) * 32 +
-                          kLongCap * 8 + kLongRows * 4;   // records, exchange, slot records, longer rows
+    // weights (+ bias), positions, exchange words, slot records field by field, longer rows
+    const int64_t fixed = int64_t(HAS_BETA ? 8 : 4) * C + 2 * C + (MAXW / G) * 8 * G * 4 + int64_t(slot_room) * 12 +
+                          int64_t(other_room) * 12 + kLongRows * 16 + kLongCap * 8;
     int tok_fit = int((kSmemBudget - fixed) / (int64_t(row_words) * 4));
     if (tok_fit > MAXW / G) tok_fit = MAXW / G;
     if (share_sm) {
@@ -767,7 +805,7 @@ int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage&
     if (W < 4) W = 4;                                       // spare warps help copy the records
     const size_t smem = size_t(fixed) + size_t(tok) * row_words * 4;
     QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    kern<<<grid, 32 * W, smem, st>>>(static_cast<const __nv_bfloat16*>(x), M, eps, bits, im, row_words, tok, rm,
+    kern<<<grid, 32 * W, smem, st>>>(static_cast<const __nv_bfloat16*>(x), M, eps, bits, im, row_words, other_room, tok, rm,
                                      codes, a_scale, a_zero, a_rowsum);
     return after_launch();
 }
@@ -791,9 +829,10 @@ int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage&
 
 template <int NPL, int G, int MAXW>
 int launch_token_variant(bool has_beta, bool packed, const void* x, int64_t M, float eps, int bits,
-                         const WarpImage& im, int slot_room, const RawMap& rm, uint8_t* codes, float* a_scale,
+                         const WarpImage& im, int slot_room, int other_room, const RawMap& rm, uint8_t* codes,
+                         float* a_scale,
                          float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool share_sm) {
-#define QLLM_RQT(B, P) launch_token<NPL, G, B, P, MAXW>(x, M, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm)
+#define QLLM_RQT(B, P) launch_token<NPL, G, B, P, MAXW>(x, M, eps, bits, im, slot_room, other_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm)
     if (has_beta) return packed ? QLLM_RQT(true, true) : QLLM_RQT(true, false);
     return packed ? QLLM_RQT(false, true) : QLLM_RQT(false, false);
 #undef QLLM_RQT
@@ -816,16 +855,22 @@ int compile_reassemble_map(int C, const float* gamma, const float* beta, const i
                            const float* coef, void* image, cudaStream_t st) {
     if (!warp_kernel_serves(C)) return QLLM_ERR_UNSUPPORTED;
     const WarpImage im = warp_image_at(image, C);
-    QLLM_CUDA_TRY(cudaMemsetAsync(im.head, 0, 16, st));
+    QLLM_CUDA_TRY(cudaMemsetAsync(im.head, 0, 32, st));
+    count_rows_kernel<<<(C + 255) / 256, 256, 0, st>>>(C, ptr, im);
     compile_map_warp_kernel<<<(C + 255) / 256, 256, 0, st>>>(C, gamma, beta, ptr, src, coef, im);
-    return after_launch();
+    return after_launch(2);
 }
 
 int reassemble_map_slots(int C, const void* image, cudaStream_t st, int* slots) {
     if (!warp_kernel_serves(C)) return QLLM_ERR_UNSUPPORTED;
     const WarpImage im = warp_image_at(const_cast<void*>(image), C);
-    QLLM_CUDA_TRY(cudaMemcpyAsync(slots, im.head, sizeof(int), cudaMemcpyDeviceToHost, st));
+    int head[8];
+    QLLM_CUDA_TRY(cudaMemcpyAsync(head, im.head, sizeof(head), cudaMemcpyDeviceToHost, st));
     QLLM_CUDA_TRY(cudaStreamSynchronize(st));
+    // rows with two entries + rows with more, and the latter again in the upper half; -1 (unknown: the launcher
+    // then assumes the largest image) when the image's slots cannot serve a launch anyway
+    const bool fits = head[4] + head[5] <= kSlotCap && head[5] <= kOtherCap && head[6] <= kLongRows;
+    *slots = fits ? ((head[5] << 16) | (head[4] + head[5])) : -1;
     return QLLM_OK;
 }
 
@@ -850,13 +895,19 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
         slots_known = -1;
     }
     const WarpImage im = warp_image_at(const_cast<void*>(map_image), C);
-    int slot_room = kSlotCap;
-    if (slots_known >= 0) slot_room = slots_known > kSlotCap ? 0 : ((slots_known + 3) & ~3);
+    // room for slot records and slot values: exact when the caller knows the image's counts, else the largest
+    // image's total with a quarter of it for rows of three and more entries (an image beyond the room makes the
+    // launch walk the CSR arrays)
+    int slot_room = kSlotCap, other_room = kSlotCap / 4;
+    if (slots_known >= 0) {
+        slot_room = ((slots_known & 0xFFFF) + 3) & ~3;
+        other_room = ((slots_known >> 16) + 3) & ~3;
+    }
     const RawMap rm{gamma, ptr, src, coef};
     const bool packed = bits == 4 && !byte_lanes, has_beta = beta != nullptr;
     if (x_dtype == QLLM_BF16) {
         // LLaMA hidden sizes: shape fixed at compile time
-#define QLLM_TOKEN_ARGS has_beta, packed, x, M, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm
+#define QLLM_TOKEN_ARGS has_beta, packed, x, M, eps, bits, im, slot_room, other_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm
         if (M <= device_sm_count()) {                          // one token per CTA: spread it over more warps
             if (C == 4096) return launch_token_variant<16, 8, 8>(QLLM_TOKEN_ARGS);
             if (C == 5120) return launch_token_variant<40, 4, 4>(QLLM_TOKEN_ARGS);
