@@ -367,6 +367,7 @@ reassemble_quant_warp(const XT* __restrict__ x, int64_t M, int C, float eps, int
             }
             d[C + vi] = e;
         }
+        if (nlong > 0) __syncwarp();                           // another lane wrote this slot's record value just above
         for (int k = lane; k < nlong; k += 32) {               // the few rows longer than a record
             const int4 lm = __ldg(im.lmeta + k);
             d[C + lm.x] = lm.w ? pair_row(im.lent, d, lm.y, lm.z) : csr_row(rm, d, C, lm.y, lm.z);
@@ -624,6 +625,7 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
                 }
                 d[C + vi] = e;
             }
+            if (nlong > 0) token_sync<G>(barid);           // another lane wrote this slot's record value just above
             for (int k = g0; k < nlong; k += GS) {         // few rows
                 const int4 lm = s_lmeta[k];
                 d[C + lm.x] = lm.w ? pair_row(s_lent, d, lm.y, lm.z) : csr_row(rm, d, C, lm.y, lm.z);

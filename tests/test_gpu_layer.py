@@ -126,5 +126,7 @@ def test_layer_full_size_two_halves_sampled(name):
     xh = torch.from_numpy(x.view(np.int16)).pin_memory()
     oh = torch.zeros((M, N), dtype=torch.bfloat16).pin_memory()
     layer.forward_host(xh, oh, M)
-    assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
+    diff = oh.view(torch.int16) != out.cpu().view(torch.int16)
+    assert not bool(diff.any()), (f"{int(diff.sum())} entries differ, rows {torch.nonzero(diff.any(1)).flatten()[:8].tolist()}"
+                                  f" cols {torch.nonzero(diff.any(0)).flatten()[:8].tolist()}")
     layer.destroy()
