@@ -177,6 +177,9 @@ struct qllm_layer {
     cudaEvent_t ev_start = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
     const uint8_t* w_ready = nullptr;            // expanded weights in flight / ready for the next GEMM call
     int64_t w_ready_M = -1;
+    // a host-buffer call in chunks expands the weights for its first chunk only: the later chunks read the same bytes
+    bool hold_w = false;
+    const uint8_t* held_w = nullptr;
     // 4-bit activations of a call that will take the byte-lane GEMM are written one code per byte by the
     // pre-GEMM kernel itself (no expansion pass): lane width of the codes now in the workspace
     int lane_bits = 0;
@@ -345,11 +348,14 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
         uint8_t* buf = nullptr;
         int rc = stream_scratch(kScratchExpand, st, a_bytes + w_bytes, &buf);
         if (rc != QLLM_OK) return rc;
-        QLLM_CUDA_TRY(cudaEventRecord(L->ev_fork, st));           // earlier users of the scratch are done
-        QLLM_CUDA_TRY(cudaStreamWaitEvent(L->side, L->ev_fork, 0));
-        rc = launch_expand_codes(L->w_codes, L->N, L->C, buf + a_bytes, L->side);
-        if (rc != QLLM_OK) return rc;
-        QLLM_CUDA_TRY(cudaEventRecord(L->ev_join, L->side));
+        if (!(L->hold_w && L->held_w == buf + a_bytes)) {
+            QLLM_CUDA_TRY(cudaEventRecord(L->ev_fork, st));       // earlier users of the scratch are done
+            QLLM_CUDA_TRY(cudaStreamWaitEvent(L->side, L->ev_fork, 0));
+            rc = launch_expand_codes(L->w_codes, L->N, L->C, buf + a_bytes, L->side);
+            if (rc != QLLM_OK) return rc;
+            QLLM_CUDA_TRY(cudaEventRecord(L->ev_join, L->side));
+            if (L->hold_w) L->held_w = buf + a_bytes;
+        }
         L->w_ready = buf + a_bytes;
         L->w_ready_M = M;
     }
@@ -423,16 +429,23 @@ int qllm_layer_forward_host(qllm_layer_t* L, const void* x_host, int64_t M, void
     }
     int rc = QLLM_OK;
     nk = 0;
+    L->hold_w = true;                                              // one weight expansion serves all chunks
+    L->held_w = nullptr;
     for (int64_t m0 = 0; m0 < M && rc == QLLM_OK; m0 += rows, ++nk) {
         const int64_t mk = std::min<int64_t>(rows, M - m0);
-        QLLM_CUDA_TRY(cudaStreamWaitEvent(st, L->ev_in[nk], 0));
+        cudaError_t e = cudaStreamWaitEvent(st, L->ev_in[nk], 0);
+        if (e != cudaSuccess) { rc = cuda_fail(e); break; }
         rc = qllm_layer_forward(L, xd + size_t(m0) * L->C * xb, mk, od + size_t(m0) * L->N * ob, stream);
         if (rc != QLLM_OK) break;
-        QLLM_CUDA_TRY(cudaEventRecord(L->ev_done[nk], st));
-        QLLM_CUDA_TRY(cudaStreamWaitEvent(L->d2h, L->ev_done[nk], 0));
-        QLLM_CUDA_TRY(cudaMemcpyAsync(oh + size_t(m0) * L->N * ob, od + size_t(m0) * L->N * ob, size_t(mk) * L->N * ob,
-                                      cudaMemcpyDeviceToHost, L->d2h));
+        e = cudaEventRecord(L->ev_done[nk], st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(L->d2h, L->ev_done[nk], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(oh + size_t(m0) * L->N * ob, od + size_t(m0) * L->N * ob, size_t(mk) * L->N * ob,
+                                cudaMemcpyDeviceToHost, L->d2h);
+        if (e != cudaSuccess) { rc = cuda_fail(e); break; }
     }
+    L->hold_w = false;
+    L->held_w = nullptr;
     // nothing of this call may be in flight when it returns, whatever happened
     const cudaError_t e1 = cudaStreamSynchronize(L->h2d), e2 = cudaStreamSynchronize(st), e3 = cudaStreamSynchronize(L->d2h);
     if (rc != QLLM_OK) return rc;
