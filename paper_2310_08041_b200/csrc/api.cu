@@ -24,7 +24,7 @@ int* device_status_word() {
 
 namespace {
 std::mutex g_scratch_mu;
-struct StreamScratch { cudaStream_t st; uint8_t* ptr; size_t cap; };
+struct StreamScratch { cudaStream_t st; uint8_t* ptr; size_t cap; uint64_t epoch; cudaEvent_t done; };
 std::vector<StreamScratch> g_stream_scratch[kScratchKinds][64];
 }  // namespace
 
@@ -40,6 +40,40 @@ int device_sm_count() {
     return n;
 }
 
+// Writers of a stream's scratch (the stream itself, or a layer's side stream working ahead for it) take turns:
+// scratch_write_begin makes `writer` wait for the previous writer, scratch_write_end records the new contents'
+// completion and returns their version.  A holder of data in the scratch (a layer whose expanded weights wait
+// there for its GEMM call) compares versions (scratch_version) to see whether the data is still its own.
+static StreamScratch* find_scratch(int kind, cudaStream_t st) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || kind < 0 || kind >= kScratchKinds) return nullptr;
+    for (auto& x : g_stream_scratch[kind][dev])
+        if (x.st == st) return &x;
+    return nullptr;
+}
+int scratch_write_begin(int kind, cudaStream_t st, cudaStream_t writer) {
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    StreamScratch* e = find_scratch(kind, st);
+    if (!e) return QLLM_ERR_UNSUPPORTED;
+    if (!e->done) QLLM_CUDA_TRY(cudaEventCreateWithFlags(&e->done, cudaEventDisableTiming));
+    QLLM_CUDA_TRY(cudaStreamWaitEvent(writer, e->done, 0));     // no-op until a writer has recorded it
+    return QLLM_OK;
+}
+int scratch_write_end(int kind, cudaStream_t st, cudaStream_t writer, uint64_t* version) {
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    StreamScratch* e = find_scratch(kind, st);
+    if (!e || !e->done) return QLLM_ERR_UNSUPPORTED;
+    QLLM_CUDA_TRY(cudaEventRecord(e->done, writer));
+    ++e->epoch;
+    if (version) *version = e->epoch;
+    return QLLM_OK;
+}
+uint64_t scratch_version(int kind, cudaStream_t st) {
+    std::lock_guard<std::mutex> lk(g_scratch_mu);
+    StreamScratch* e = find_scratch(kind, st);
+    return e ? e->epoch : 0;
+}
+
 int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out) {
     int dev = 0;
     QLLM_CUDA_TRY(cudaGetDevice(&dev));
@@ -47,12 +81,13 @@ int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out) {
     std::lock_guard<std::mutex> lk(g_scratch_mu);
     StreamScratch* e = nullptr;
     for (auto& x : g_stream_scratch[kind][dev]) if (x.st == st) e = &x;
-    if (!e) { g_stream_scratch[kind][dev].push_back({st, nullptr, 0}); e = &g_stream_scratch[kind][dev].back(); }
+    if (!e) { g_stream_scratch[kind][dev].push_back({st, nullptr, 0, 0, nullptr}); e = &g_stream_scratch[kind][dev].back(); }
     if (e->cap < bytes) {
         if (e->ptr) QLLM_CUDA_TRY(cudaFree(e->ptr));
         e->ptr = nullptr; e->cap = 0;
         QLLM_CUDA_TRY(cudaMalloc(&e->ptr, bytes));
         e->cap = bytes;
+        ++e->epoch;
     }
     *out = e->ptr;
     return QLLM_OK;
@@ -115,9 +150,13 @@ int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, i
             uint8_t* buf = nullptr;
             int rc = stream_scratch(kScratchExpand, st, a_bytes + w_bytes, &buf);
             if (rc != QLLM_OK) return rc;
+            const bool reuse_w = wp && w_ready == buf + a_bytes;
+            const bool writes = ap || (wp && !reuse_w);
+            if (writes) { rc = scratch_write_begin(kScratchExpand, st, st); if (rc != QLLM_OK) return rc; }
             if (ap) { rc = launch_expand_codes(a, M, K, buf, st); if (rc != QLLM_OK) return rc; a = buf; }
-            if (wp && w_ready == buf + a_bytes) w = w_ready;
+            if (reuse_w) w = w_ready;
             else if (wp) { rc = launch_expand_codes(w, N, K, buf + a_bytes, st); if (rc != QLLM_OK) return rc; w = buf + a_bytes; }
+            if (writes) { rc = scratch_write_end(kScratchExpand, st, st, nullptr); if (rc != QLLM_OK) return rc; }
             return launch_qgemm_tc(a, w, M, N, K, 8, 8, ep, st);
         }
         return launch_qgemm_tc(a, w, M, N, K, a_bits, w_bits, ep, st);
@@ -177,6 +216,7 @@ struct qllm_layer {
     cudaEvent_t ev_start = nullptr, ev_in[kHostChunks] = {}, ev_done[kHostChunks] = {};
     const uint8_t* w_ready = nullptr;            // expanded weights in flight / ready for the next GEMM call
     int64_t w_ready_M = -1;
+    uint64_t w_epoch = 0;                        // version of the scratch contents when they were written
     // a host-buffer call in chunks expands the weights for its first chunk only: the later chunks read the same bytes
     bool hold_w = false;
     const uint8_t* held_w = nullptr;
@@ -348,12 +388,17 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
         uint8_t* buf = nullptr;
         int rc = stream_scratch(kScratchExpand, st, a_bytes + w_bytes, &buf);
         if (rc != QLLM_OK) return rc;
-        if (!(L->hold_w && L->held_w == buf + a_bytes)) {
+        if (!(L->hold_w && L->held_w == buf + a_bytes &&
+              scratch_version(kScratchExpand, st) == L->w_epoch)) {
             QLLM_CUDA_TRY(cudaEventRecord(L->ev_fork, st));       // earlier users of the scratch are done
             QLLM_CUDA_TRY(cudaStreamWaitEvent(L->side, L->ev_fork, 0));
+            rc = scratch_write_begin(kScratchExpand, st, L->side);  // another layer may be expanding there
+            if (rc != QLLM_OK) return rc;
             rc = launch_expand_codes(L->w_codes, L->N, L->C, buf + a_bytes, L->side);
             if (rc != QLLM_OK) return rc;
             QLLM_CUDA_TRY(cudaEventRecord(L->ev_join, L->side));
+            rc = scratch_write_end(kScratchExpand, st, L->side, &L->w_epoch);
+            if (rc != QLLM_OK) return rc;
             if (L->hold_w) L->held_w = buf + a_bytes;
         }
         L->w_ready = buf + a_bytes;
@@ -368,7 +413,10 @@ int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {
     if (!L || !out) return QLLM_ERR_NULL;
     if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
     const uint8_t* w_ready = nullptr;
-    if (L->w_ready && L->w_ready_M == M) {
+    if (L->w_ready && L->w_ready_M == M &&
+        scratch_version(kScratchExpand, static_cast<cudaStream_t>(stream)) == L->w_epoch) {
+        // the expanded weights are still this layer's (another layer or a direct call on the stream would have
+        // bumped the version); otherwise the GEMM call expands them again itself
         QLLM_CUDA_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), L->ev_join, 0));
         w_ready = L->w_ready;
     }

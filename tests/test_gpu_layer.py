@@ -130,3 +130,35 @@ def test_layer_full_size_two_halves_sampled(name):
     assert not bool(diff.any()), (f"{int(diff.sum())} entries differ, rows {torch.nonzero(diff.any(1)).flatten()[:8].tolist()}"
                                   f" cols {torch.nonzero(diff.any(0)).flatten()[:8].tolist()}")
     layer.destroy()
+
+
+def test_two_layers_interleaved_on_one_stream():
+    """The byte expansion of 4-bit weights lives in scratch memory shared by everything on a stream.  Two layers
+    whose half-step calls interleave (A pre-GEMM, B pre-GEMM, A GEMM, B GEMM) must each still multiply with their
+    own weights, exactly as when they run one after the other."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    layers, xs, refs = [], [], []
+    for seed, N in ((31, 256), (32, 384)):
+        cfg = synth.CONFIGS["c2"].scaled(M=520, K=512, N=N, n_outlier=4, seed=seed)
+        L = parity.oracle_layer(cfg)
+        h = B.qllm_build_reassembly(L["absmax"], L["theta"], L["W"], L["lrA"], L["lrB"], cfg.w_bits)
+        layer = B.Layer(h, L["gamma"], L["beta"], cfg.ln_eps, None, cfg.a_bits, B.QLLM_BF16, B.QLLM_F32, max_M=cfg.M)
+        x = G.dev_x(synth.activations(cfg))
+        ref = torch.zeros((cfg.M, N), dtype=torch.float32, device=G.DEV)
+        layer.forward(x, ref)
+        layers.append(layer); xs.append(x); refs.append(ref)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        outs = [torch.zeros_like(r) for r in refs]
+        layers[0].reassemble_quant(xs[0])
+        layers[1].reassemble_quant(xs[1])
+        layers[0].qgemm(xs[0].shape[0], outs[0])
+        layers[1].qgemm(xs[1].shape[0], outs[1])
+        torch.cuda.synchronize()
+        assert B.qllm_poll_status() == 0
+        # each layer's workspace is its own, so the activations are right either way; the weights are what is shared
+        assert torch.equal(outs[0], refs[0]) and torch.equal(outs[1], refs[1])
+    for layer in layers:
+        layer.destroy()
