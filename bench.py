@@ -65,7 +65,11 @@ class ClockSampler:
             return None
         time.sleep(0.15)
         self.proc.terminate()
-        rows = [r for ts, r in self.rows if t0 <= ts <= t1 + 0.2] or [r for _, r in self.rows]
+        timed = [r for ts, r in self.rows if t0 <= ts <= t1]
+        # a short timed region sees few 100 ms samples: then every sample since the warm-up began counts
+        # (the same kernels ran throughout), and the line says so
+        rows = timed if len(timed) >= 3 else [r for _, r in self.rows]
+        window = "timed steps" if len(timed) >= 3 else "warm-up + timed steps + end-to-end steps"
         if not rows:
             return None
         sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
@@ -73,7 +77,7 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = sorted({n for r in rows for n, v in zip(names, r[3:7]) if v.lower().startswith("active")})
         return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
-                    reasons=reasons, samples=len(rows))
+                    reasons=reasons, samples=len(rows), samples_in_timed_steps=len(timed), window=window)
 
 
 def _oracle_sample(cfg, rows, L=None):
@@ -101,7 +105,7 @@ def run_reference(args):
         return
     cfg = synth.CONFIGS[args.workload]
     # bounded sample per step so that the whole run ends within a few minutes (~45 rows/s)
-    rows = args.ref_rows or max(8, min(512, 5400 // max(1, args.steps + args.warmup)))
+    rows = args.ref_rows or max(1, min(512, 7000 // max(1, args.steps + args.warmup)))
     L = None
     for _ in range(min(args.warmup, 1)):
         _, _, L = _oracle_sample(cfg, max(1, rows // 8), L)
@@ -182,12 +186,12 @@ def run_gpu(args):
         if evs:
             evs[2].record()
 
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(args.warmup):
         flush.zero_()
         step()
     barrier()
     assert B.qllm_poll_status() == 0, "device-side wait timed out during warm-up"
-    sampler = ClockSampler(local) if rank == 0 else None
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     n0 = B.qllm_launch_count()
     barrier()
@@ -198,7 +202,6 @@ def run_gpu(args):
     barrier()
     t_end = time.time()
     launches = B.qllm_launch_count() - n0
-    clocks = sampler.stop(t_start, t_end) if sampler else None
     assert B.qllm_poll_status() == 0, "device-side wait timed out"
     t_pre = [e[0].elapsed_time(e[1]) for e in events]
     t_gemm = [e[1].elapsed_time(e[2]) for e in events]
@@ -219,6 +222,7 @@ def run_gpu(args):
         e2e_ev[i][1].record()
     barrier()
     ms_e2e = sum(a.elapsed_time(b) for a, b in e2e_ev) / e2e_steps
+    clocks = sampler.stop(t_start, t_end) if sampler else None
     h2d = M * K * (2 if cfg.x_dtype == "bf16" else 4)
     d2h = M * N * 2
 
@@ -287,8 +291,8 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c2_w4a8"])
     ap.add_argument("--ref-rows", type=int, default=0, help="token rows of the oracle sample (0 = auto)")
