@@ -282,7 +282,13 @@ int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const f
                       float ln_eps, const float* bias, int a_bits, int x_dtype, int out_dtype,
                       int64_t max_M, qllm_layer_t** out);
 void qllm_layer_destroy(qllm_layer_t* layer);
-/* x, out: device.  Asynchronous on stream. */
+/* x, out: device.  Asynchronous on stream.
+ * Stream capture: once a call of the same M has run on the stream (scratch sized, kernel attributes set), a
+ * later call issues only capturable work -- kernel launches and the event fork/join of the internal stream
+ * that expands 4-bit weights -- so it may be recorded into a CUDA graph.  The graph holds the scratch
+ * pointers of that moment: create every layer that will run on the stream, and run each once at its largest
+ * M, before capturing.  Capture whole forwards (both halves inside the capture or both outside it), and do
+ * not replay a graph between the two half-step calls of another layer on the same stream. */
 int qllm_layer_forward(qllm_layer_t* layer, const void* x, int64_t M, void* out, void* stream);
 /* The two halves of qllm_layer_forward, for callers that time or schedule them separately:
  * qllm_layer_reassemble_quant runs the fused pre-GEMM kernel on x[M][C] (device) into the layer's

@@ -24,7 +24,17 @@ int* device_status_word() {
 
 namespace {
 std::mutex g_scratch_mu;
-struct StreamScratch { cudaStream_t st; uint8_t* ptr; size_t cap; uint64_t epoch; cudaEvent_t done; };
+struct StreamScratch {
+    cudaStream_t st; uint8_t* ptr; size_t cap; uint64_t epoch; cudaEvent_t done;
+    unsigned long long done_capture;   // id of the stream capture `done` was last recorded in, 0 = outside any
+};
+// Id of the capture `st` is part of, 0 when it is not capturing.
+unsigned long long capture_id(cudaStream_t st) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    unsigned long long id = 0;
+    if (cudaStreamGetCaptureInfo(st, &cs, &id) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return cs == cudaStreamCaptureStatusActive ? id : 0;
+}
 std::vector<StreamScratch> g_stream_scratch[kScratchKinds][64];
 }  // namespace
 
@@ -56,7 +66,10 @@ int scratch_write_begin(int kind, cudaStream_t st, cudaStream_t writer) {
     StreamScratch* e = find_scratch(kind, st);
     if (!e) return QLLM_ERR_UNSUPPORTED;
     if (!e->done) QLLM_CUDA_TRY(cudaEventCreateWithFlags(&e->done, cudaEventDisableTiming));
-    QLLM_CUDA_TRY(cudaStreamWaitEvent(writer, e->done, 0));     // no-op until a writer has recorded it
+    // no-op until a writer has recorded it.  An event recorded inside a stream capture cannot be waited on
+    // from outside it, nor the reverse: across that boundary the writers are ordered by the stream itself
+    // (the graph runs in stream order, after the work issued before it)
+    if (capture_id(writer) == e->done_capture) QLLM_CUDA_TRY(cudaStreamWaitEvent(writer, e->done, 0));
     return QLLM_OK;
 }
 int scratch_write_end(int kind, cudaStream_t st, cudaStream_t writer, uint64_t* version) {
@@ -64,6 +77,7 @@ int scratch_write_end(int kind, cudaStream_t st, cudaStream_t writer, uint64_t* 
     StreamScratch* e = find_scratch(kind, st);
     if (!e || !e->done) return QLLM_ERR_UNSUPPORTED;
     QLLM_CUDA_TRY(cudaEventRecord(e->done, writer));
+    e->done_capture = capture_id(writer);
     ++e->epoch;
     if (version) *version = e->epoch;
     return QLLM_OK;
@@ -81,7 +95,7 @@ int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out) {
     std::lock_guard<std::mutex> lk(g_scratch_mu);
     StreamScratch* e = nullptr;
     for (auto& x : g_stream_scratch[kind][dev]) if (x.st == st) e = &x;
-    if (!e) { g_stream_scratch[kind][dev].push_back({st, nullptr, 0, 0, nullptr}); e = &g_stream_scratch[kind][dev].back(); }
+    if (!e) { g_stream_scratch[kind][dev].push_back({st, nullptr, 0, 0, nullptr, 0}); e = &g_stream_scratch[kind][dev].back(); }
     if (e->cap < bytes) {
         if (e->ptr) QLLM_CUDA_TRY(cudaFree(e->ptr));
         e->ptr = nullptr; e->cap = 0;

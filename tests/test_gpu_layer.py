@@ -162,3 +162,46 @@ def test_two_layers_interleaved_on_one_stream():
         assert torch.equal(outs[0], refs[0]) and torch.equal(outs[1], refs[1])
     for layer in layers:
         layer.destroy()
+
+
+def test_forward_under_stream_capture():
+    """qllm_layer_forward issues only capturable work once its buffers are warm (launches, and the fork/join
+    of the side stream that expands 4-bit weights): a CUDA graph of two layers replays to the same bits as the
+    direct calls, before and after other direct calls on the stream."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    layers, xs, refs = [], [], []
+    for seed, N in ((41, 256), (42, 384)):
+        cfg = synth.CONFIGS["c2"].scaled(M=520, K=512, N=N, n_outlier=4, seed=seed)
+        L = parity.oracle_layer(cfg)
+        h = B.qllm_build_reassembly(L["absmax"], L["theta"], L["W"], L["lrA"], L["lrB"], cfg.w_bits)
+        layers.append(B.Layer(h, L["gamma"], L["beta"], cfg.ln_eps, None, cfg.a_bits, B.QLLM_BF16, B.QLLM_F32,
+                              max_M=cfg.M))
+        xs.append(G.dev_x(synth.activations(cfg)))
+        refs.append(torch.zeros((cfg.M, N), dtype=torch.float32, device=G.DEV))
+    s = torch.cuda.Stream()
+    outs = [torch.zeros_like(r) for r in refs]
+    with torch.cuda.stream(s):
+        for layer, x, ref in zip(layers, xs, refs):      # warm: scratch sized, attributes set
+            layer.forward(x, ref)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        for layer, x, out in zip(layers, xs, outs):
+            layer.forward(x, out)
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for o in outs:
+            o.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert B.qllm_poll_status() == 0
+        assert torch.equal(outs[0], refs[0]) and torch.equal(outs[1], refs[1]), rep
+        with torch.cuda.stream(s):                        # a direct call between replays
+            chk = torch.zeros_like(refs[rep % 2])
+            layers[rep % 2].forward(xs[rep % 2], chk)
+        torch.cuda.synchronize()
+        assert torch.equal(chk, refs[rep % 2])
+    for layer in layers:
+        layer.destroy()
