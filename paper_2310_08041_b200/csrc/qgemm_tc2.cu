@@ -10,12 +10,13 @@
 // settles near 150.
 // Roles per CTA: warp 0 TMA producer (own halves), warp 1 MMA issuer (one thread of the leader
 // CTA, cluster rank 0, issues for the pair) and owner of the tensor-memory allocation,
-// warps 2-5 epilogue (own 128 rows).  No TMA multicast is used.
+// warps 2-9 epilogue (own 128 rows; two warps per quarter of the TMEM lanes take alternate 32-column
+// chunks, stage them in shared memory and hand them to the copy engine).  No TMA multicast is used.
 //
 // Barriers:  full[s]      (leader's)  bytes of both CTAs' tiles of stage s have landed
 //            empty[s]     (own CTA)   the pair's MMAs that read stage s are complete
 //            acc_full[b]  (own CTA)   accumulator buffer b is complete
-//            acc_empty[b] (leader's)  8 arrivals: the 4 epilogue warps of each CTA drained buffer b
+//            acc_empty[b] (leader's)  16 arrivals: the 8 epilogue warps of each CTA drained buffer b
 // The leader's MMA thread commits to the barriers of both CTAs.  Every wait is bounded (see
 // wait_bounded); the pair leaves together through a cluster barrier.
 
@@ -47,11 +48,13 @@ struct PairTile {
     static constexpr int SUBA = BM * BK, SUBW = HALF_N * BK;    // one swizzled 128-byte-wide sub-tile
     static constexpr int OPA = KS * SUBA, OPW = KS * SUBW;
     static constexpr int STAGE = OPA + OPW;
-    static constexpr int FIXED = BN * 16 + 256;                 // column terms + barriers
+    static constexpr int EPI_WARPS = 8;                         // two per quarter of the TMEM lanes, alternating chunks
+    static constexpr int OUTBUF = EPI_WARPS * 2048;             // per epilogue warp: one 32-row x 64-byte store box
+    static constexpr int FIXED = BN * 16 + 256 + OUTBUF;        // column terms + barriers + store staging
     static constexpr int FIT = (227 * 1024 - 1024 - FIXED) / STAGE;
     static constexpr int STAGES = FIT > 8 ? 8 : FIT;
     static constexpr int SMEM = STAGES * STAGE + FIXED + 1024;  // + alignment slack
-    static constexpr int THREADS = 32 * kFirstUnpackWarp;       // 6 warps
+    static constexpr int THREADS = 32 * (kFirstEpiWarp + EPI_WARPS);   // 10 warps
     static constexpr uint32_t TMEM_COLS = 2 * BN <= 256 ? 256 : 512;
     static_assert(HALF_N % 8 == 0 && BN % 16 == 0 && BN <= 256, "tile width");
 };
@@ -59,14 +62,15 @@ struct PairTile {
 template <int BN>
 __global__ void __launch_bounds__(PairTile<BN>::THREADS, 1)
 qgemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-                 int64_t M, int N, int K, EpilogueArgs ep, int* status) {
+                 const __grid_constant__ CUtensorMap tmO, int64_t M, int N, int K, EpilogueArgs ep, int* status) {
     using T = PairTile<BN>;
     constexpr int S = T::STAGES;
     extern __shared__ uint8_t smem_dyn[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
     uint8_t* opA = smem;
     uint8_t* opW = opA + S * T::OPA;
-    int4* colterm = reinterpret_cast<int4*>(opW + S * T::OPW);
+    uint8_t* outbuf = opW + S * T::OPW;                         // 1024-byte aligned (stages are multiples of 1024)
+    int4* colterm = reinterpret_cast<int4*>(outbuf + T::OUTBUF);
     uint64_t* bars = reinterpret_cast<uint64_t*>(colterm + BN);
     uint64_t* full = bars;                 // [S]
     uint64_t* empty = bars + S;            // [S]
@@ -91,13 +95,14 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&acc_full[b], 1);
-            ptx::mbar_init(&acc_empty[b], 8);
+            ptx::mbar_init(&acc_empty[b], 2 * T::EPI_WARPS);
         }
         *abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
         ptx::prefetch_tensormap(&tmA);
         ptx::prefetch_tensormap(&tmW);
+        ptx::prefetch_tensormap(&tmO);
     }
     __syncthreads();
     ptx::cluster_sync();                    // both CTAs' barriers exist before any remote arrive
@@ -185,36 +190,60 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     } else {
         // ------------------------------------------------------------------ epilogue (own 128 rows)
         const int quad = warp & 3;                        // TMEM lanes 32*quad .. +31
-        const int et = threadIdx.x - 32 * kFirstEpiWarp;  // 0..127
+        const int half = (warp - kFirstEpiWarp) >> 2;     // even or odd 32-column chunks of the tile
+        const int et = threadIdx.x - 32 * kFirstEpiWarp;  // 0 .. 32 * EPI_WARPS - 1
+        constexpr int ET = 32 * T::EPI_WARPS;
         const uint32_t accempty_addr[2] = {ptx::map_to_cta(ptx::smem_addr(&acc_empty[0]), 0),
                                            ptx::map_to_cta(ptx::smem_addr(&acc_empty[1]), 0)};
+        uint8_t* mybuf = outbuf + (warp - kFirstEpiWarp) * 2048;
         uint32_t lt = 0;
         for (int tile = pair; tile < num_tiles; tile += npairs, ++lt) {
             const uint32_t abuf = lt & 1, aph = (lt >> 1) & 1;
             const int m0 = (tile % tiles_m) * 2 * BM + int(rank) * BM;
             const int n0 = (tile / tiles_m) * BN;
-            ptx::named_bar_sync(1, 128);
-            stage_col_terms(ep, colterm, BN, n0, N, K, et, 128);
-            ptx::named_bar_sync(1, 128);
-            const int64_t m = int64_t(m0) + quad * 32 + lane;
-            RowTerm rt{0.f, 0, 0};
-            if (!ep.raw_acc && m < M) rt = make_row_term(ep.a_scale, ep.a_zero, ep.a_rowsum, m);
+            ptx::named_bar_sync(1, ET);
+            stage_col_terms(ep, colterm, BN, n0, N, K, et, ET);
+            ptx::named_bar_sync(1, ET);
+            const int row0 = m0 + quad * 32;              // first of this warp's 32 rows; rows >= M are not written
+            RowTerm rt[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int64_t m = int64_t(row0) + (lane >> 2) + 8 * i;
+                rt[i] = RowTerm{0.f, 0, 0};
+                if (!ep.raw_acc && m < M) rt[i] = make_row_term(ep.a_scale, ep.a_zero, ep.a_rowsum, m);
+            }
             if (!wait_bounded(&acc_full[abuf], aph, ab)) break;
             ptx::tc_fence_after_sync();
 #pragma unroll 1
-            for (int ch = 0; ch < BN / 32; ++ch) {
+            for (int ch = half; ch < BN / 32; ch += 2) {
                 const int nb = n0 + ch * 32;
-                if (nb >= N) break;                       // uniform over the CTA
-                uint32_t r[32];
-                ptx::tmem_ld_32x32b_x32(tmem_base + (uint32_t(quad * 32) << 16) + abuf * BN + ch * 32, r);
+                if (nb >= N) break;                       // uniform over the warp
+                uint32_t lo[16], hi[16];
+                const uint32_t taddr = tmem_base + (uint32_t(quad * 32) << 16) + abuf * BN + ch * 32;
+                ptx::tmem_ld_16x256b_x4(taddr, lo);
+                ptx::tmem_ld_16x256b_x4(taddr + (16u << 16), hi);
                 ptx::tmem_ld_wait();
-                if (m < M) store_chunk(ep, r, colterm + ch * 32, rt, m, N, nb);
-                __syncwarp();   // reconverge before the next warp-wide TMEM load
+                stage_chunk(ep, lo, hi, colterm + ch * 32, rt, lane, nb,
+                            [&](int) {
+                                // the previous box used this buffer: its shared-memory reads must be over
+                                if (lane == 0) ptx::bulk_wait_group_read<0>();
+                                __syncwarp();
+                                return mybuf;
+                            },
+                            [&](int, int x_bytes) {
+                                ptx::fence_proxy_async_smem();
+                                __syncwarp();
+                                if (lane == 0 && row0 < M) {
+                                    ptx::tma_store_2d(&tmO, mybuf, x_bytes, row0);
+                                    ptx::bulk_commit_group();
+                                }
+                            });
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(accempty_addr[abuf]);
         }
+        if (lane == 0) ptx::bulk_wait_group<0>();         // the stores are complete before the CTA retires
     }
 
     ptx::tc_fence_before_sync();
@@ -231,9 +260,10 @@ int launch_pair(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, con
                 cudaStream_t st) {
     using T = PairTile<BN>;
     static_assert(T::STAGES >= 2, "pipeline needs at least two stages");
-    CUtensorMap tmA, tmW;
+    CUtensorMap tmA, tmW, tmO;
     if (!make_map(&tmA, a, uint64_t(M), uint64_t(K), BM, BK, true) ||
-        !make_map(&tmW, w, uint64_t(N), uint64_t(K), T::HALF_N, BK, true))
+        !make_map(&tmW, w, uint64_t(N), uint64_t(K), T::HALF_N, BK, true) ||
+        !make_store_map(&tmO, ep.out, uint64_t(M), uint64_t(N) * (ep.raw_acc || ep.out_dtype == QLLM_F32 ? 4 : 2)))
         return QLLM_ERR_CUDA;
     int* status = device_status_word();
     if (!status) return QLLM_ERR_CUDA;
@@ -253,7 +283,7 @@ int launch_pair(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, con
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    QLLM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmW, M, N, K, ep, status));
+    QLLM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmW, tmO, M, N, K, ep, status));
     return after_launch();
 }
 

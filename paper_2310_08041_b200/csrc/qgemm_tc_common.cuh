@@ -118,6 +118,65 @@ __device__ __forceinline__ void store_chunk(const EpilogueArgs& ep, const uint32
     }
 }
 
+// A 32-row x 32-column chunk of the accumulator, staged for a bulk tensor store.  The values arrive in the
+// 16x256b fragment layout (lo: TMEM lanes 0..15 of the warp's quarter, hi: lanes 16..31): thread t holds rows
+// t/4 + {0, 8, 16, 24} and, per column group j, columns 8j + 2(t%4), +1 -- so it needs the terms of 8 of the
+// chunk's 32 columns instead of all of them.  (With one row per thread every thread read every column's terms:
+// 32 broadcast reads per chunk that queue behind the tensor core's operand reads in the same shared memory;
+// they took half of the epilogue's time.)  The warp's 32 rows x 64 bytes go to shared memory in the 64-byte
+// swizzle of the output tensor map (16-byte unit u of row r at unit u ^ ((r >> 1) & 3); the four rows of a
+// thread share that term), which makes the 4- and 8-byte stores of a warp conflict-free, one box per 64 bytes
+// of a row; the global writes are whole lines issued by the copy engine.
+// box(b) returns the buffer for the b-th box of this chunk (waiting until it is free), send(b, x_bytes) issues it.
+template <typename BoxFn, typename SendFn>
+__device__ __forceinline__ void stage_chunk(const EpilogueArgs& ep, const uint32_t (&lo)[16], const uint32_t (&hi)[16],
+                                            const int4* colterm, const RowTerm (&rt)[4], int lane, int nb, BoxFn box,
+                                            SendFn send) {
+    const int q = lane & 3, r0 = lane >> 2, sw = (r0 >> 1) & 3;
+    auto acc = [&](int i, int j, int e) -> uint32_t { return i < 2 ? lo[4 * j + 2 * i + e] : hi[4 * j + 2 * (i - 2) + e]; };
+    auto deq = [&](uint32_t a, const RowTerm& r, const int4& ct) -> float {
+        const int I = int(a) - ct.y * r.rowsum - r.zero * ct.z;
+        return fmaf(r.scale * __int_as_float(ct.x), float(I), __int_as_float(ct.w));
+    };
+    if (ep.raw_acc || ep.out_dtype == QLLM_F32) {
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            uint8_t* buf = box(b) + r0 * 64 + (q & 1) * 8;
+#pragma unroll
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = 2 * b + jj;
+                int4 c0 = make_int4(0, 0, 0, 0), c1 = c0;
+                if (!ep.raw_acc) { c0 = colterm[8 * j + 2 * q]; c1 = colterm[8 * j + 2 * q + 1]; }
+                const int unit = ((2 * jj + (q >> 1)) ^ sw) << 4;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint2 v;
+                    if (ep.raw_acc) {
+                        v = make_uint2(acc(i, j, 0), acc(i, j, 1));
+                    } else {
+                        v = make_uint2(__float_as_uint(deq(acc(i, j, 0), rt[i], c0)), __float_as_uint(deq(acc(i, j, 1), rt[i], c1)));
+                    }
+                    *reinterpret_cast<uint2*>(buf + i * 8 * 64 + unit) = v;
+                }
+            }
+            send(b, nb * 4 + b * 64);
+        }
+    } else {
+        uint8_t* buf = box(0) + r0 * 64 + q * 4;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int4 c0 = colterm[8 * j + 2 * q], c1 = colterm[8 * j + 2 * q + 1];
+            const int unit = (j ^ sw) << 4;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                __nv_bfloat162 v2 = __floats2bfloat162_rn(deq(acc(i, j, 0), rt[i], c0), deq(acc(i, j, 1), rt[i], c1));
+                *reinterpret_cast<uint32_t*>(buf + i * 8 * 64 + unit) = *reinterpret_cast<uint32_t*>(&v2);
+            }
+        }
+        send(0, nb * 2);
+    }
+}
+
 // Column terms of the tile's output channels -> shared memory (scale, zero, colsum - K*zero, bias).
 __device__ __forceinline__ void stage_col_terms(const EpilogueArgs& ep, int4* colterm, int bn, int n0, int N, int K,
                                                 int et, int nthreads) {
@@ -162,6 +221,19 @@ inline bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// Output matrix [rows][row_bytes] as bytes; box = 32 rows x 64 bytes in the 64-byte swizzle (stage_chunk).
+inline bool make_store_map(CUtensorMap* map, void* base, uint64_t rows, uint64_t row_bytes) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {64, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
