@@ -18,6 +18,8 @@ SHAPES = [
     (140, 272, 512, 8, 4), (33, 80, 256, 4, 8), (200, 16, 128, 4, 4), (128, 256, 128, 4, 4),
     (8, 136, 512, 6, 6), (12, 520, 1024, 8, 4), (5, 61, 256, 4, 8), (16, 22016, 4096, 4, 4), (1, 8, 128, 4, 4),
     (600, 272, 256, 4, 4), (520, 136, 512, 8, 4), (513, 80, 160, 4, 8),
+    # CTA-pair kernel edges: one row past a 128-row block, narrowest output, K that ends inside a stage, 1000^3
+    (129, 8, 128, 8, 8), (385, 264, 272, 8, 8), (1000, 1000, 1008, 6, 6),
 ]
 
 
@@ -55,7 +57,8 @@ def _epilogue_inputs(seed, M, N, a_bits, w_bits, qa, qw):
 
 @pytest.mark.parametrize("out_dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("M,N,K,a_bits,w_bits", [(5, 33, 64, 4, 4), (16, 1000, 4096, 4, 4), (130, 272, 384, 4, 4),
-                                                 (257, 528, 640, 6, 6), (9, 31, 77, 6, 6), (140, 272, 512, 8, 4)])
+                                                 (257, 528, 640, 6, 6), (9, 31, 77, 6, 6), (140, 272, 512, 8, 4),
+                                                 (385, 264, 272, 8, 8), (129, 8, 128, 8, 8)])
 def test_epilogue_matches_oracle(M, N, K, a_bits, w_bits, out_dtype):
     import torch
     import gpu_util as G
