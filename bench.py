@@ -252,7 +252,7 @@ def run_gpu(args):
                         "peak_source": f"{peaks['source']} STREAM-style copy", "ms": ms_gemm, "bytes": gemm_bytes,
                         "traffic": NCU_TRAFFIC.get((cfg.name, M))}
         else:
-            expand = (cfg.a_bits == 4 or cfg.w_bits == 4) and M >= 512
+            expand = (cfg.a_bits == 4 or cfg.w_bits == 4) and M >= 385
             roofline = {"kernel": "qllm_layer_qgemm: " + ("join of the side-stream weight expansion + " if expand and cfg.w_bits == 4 else "") +
                                   "qgemm_tc2_kernel (tcgen05 kind::i8, cta_group::2, byte lanes) + dequant epilogue",
                         "bound": "tensor", "achieved": tops, "peak": int8_peak, "unit": "TOP/s", "frac": tops / int8_peak,

@@ -119,7 +119,7 @@ int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C,
  *  K must be even when either operand is 4-bit.  |I| must fit an int32.
  *  Dispatch: M <= 16 takes a weight-streaming kernel (weights read once); larger M takes the
  *  tensor-core kernel when the shape allows it, else a plain kernel.  With a 4-bit operand and
- *  M >= 512 the 4-bit codes are first widened to byte lanes, once per call, into a second
+ *  M >= 385 the 4-bit codes are first widened to byte lanes, once per call, into a second
  *  library-owned scratch buffer kept per (device, stream) and grown with cudaMalloc like the
  *  row-sum scratch (N*K + M*K bytes at most); qllm_qgemm_noalloc never does this.
  */
@@ -305,7 +305,7 @@ int qllm_layer_forward_host(qllm_layer_t* layer, const void* x_host, int64_t M, 
 /* Borrowed DEVICE pointers of the layer's quantized-activation workspace of the last forward.
  * *lane_bits (may be NULL) receives how the codes are stored: 4 = two per byte as qllm_reassemble_quant
  * writes 4-bit codes, 8 = one per byte [M][C].  4-bit activations are stored one per byte when the
- * call's GEMM runs on byte lanes (M >= 512 on the tensor-core path): the pre-GEMM kernel then writes
+ * call's GEMM runs on byte lanes (M >= 385 on the tensor-core path): the pre-GEMM kernel then writes
  * the lanes the GEMM reads, which saves a widening pass; the code VALUES are the same. */
 int qllm_layer_workspace(qllm_layer_t* layer, uint8_t** codes, float** a_scale, float** a_zero,
                          int32_t** a_rowsum, int* lane_bits);

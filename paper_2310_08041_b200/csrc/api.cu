@@ -143,8 +143,11 @@ int check_gemm_shape(int64_t M, int N, int K, int a_bits, int w_bits) {
 
 // Token count from which expanding 4-bit operands to bytes once per call (a bandwidth-bound pre-pass
 // over N*K + M*K codes) and running the byte-lane tensor-core kernel beats unpacking every tile in
-// shared memory, which caps the tensor pipe near 40 %.
-constexpr int64_t kExpandMinM = 512;
+// shared memory, which caps the tensor pipe near 40 %: more than three 128-row blocks (measured on the 4096- and
+// 8192-channel shapes: 129-256 tokens a draw, 257-384 the in-kernel unpack wins, from 385 the expansion).
+constexpr int64_t kExpandMinM = 385;
+// Fewest tokens per chunk of a chunked host-buffer call.
+constexpr int64_t kHostChunkRows = 512;
 
 bool expand_path(int64_t M, int N, int K, int a_bits, int w_bits) {
     return M > 16 && M >= kExpandMinM && (a_bits == 4 || w_bits == 4) && qgemm_tc_supported(M, N, K, a_bits, w_bits);
@@ -393,7 +396,10 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
     if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
     L->w_ready = nullptr;
     const bool expand = expand_path(M, L->N, L->C, L->a_bits, L->w_bits);
-    const bool byte_lanes = expand && L->a_bits == 4 && reassemble_byte_lanes_supported(L->C);
+    // 4-bit activations for a tensor-core GEMM (more than 16 tokens) are written one code per byte: the GEMM
+    // then expands nothing on the activation side (below kExpandMinM tokens it unpacks only its weight tiles)
+    const bool byte_lanes = L->a_bits == 4 && M > 16 && qgemm_tc_supported(M, L->N, L->C, L->a_bits, L->w_bits) &&
+                            reassemble_byte_lanes_supported(L->C);
     L->lane_bits = (L->a_bits == 4 && !byte_lanes) ? 4 : 8;
     if (L->side && expand) {
         // start expanding the weights for the coming GEMM on the side stream: it is independent of the tokens
@@ -455,7 +461,7 @@ int qllm_layer_forward_host(qllm_layer_t* L, const void* x_host, int64_t M, void
     const size_t xb = L->x_dtype == QLLM_F32 ? 4 : 2, ob = L->out_dtype == QLLM_F32 ? 4 : 2;
     constexpr int NC = qllm_layer::kHostChunks;
     const int64_t rows = ((M + NC - 1) / NC + 127) / 128 * 128;      // tokens per chunk
-    if (rows < kExpandMinM || rows >= M) {
+    if (rows < kHostChunkRows || rows >= M) {
         // few tokens: one copy in, the path, one copy out
         QLLM_CUDA_TRY(cudaMemcpyAsync(L->x_dev, x_host, size_t(M) * L->C * xb, cudaMemcpyHostToDevice, st));
         int rc = qllm_layer_forward(L, L->x_dev, M, L->out_dev, stream);

@@ -242,23 +242,29 @@ bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits) {
 int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
                     const EpilogueArgs& ep, cudaStream_t st) {
     const bool ap = a_bits == 4, wp = w_bits == 4;
-    if (ap && wp) return launch<256, true, true>(a, w, M, N, K, ep, st);
-    if (!ap && !wp) {
-        if (qgemm_tc2_supported(M, N, K, a_bits, w_bits)) return launch_qgemm_tc2(a, w, M, N, K, ep, st);
-        // tile width that wastes the least of the last wave: cost ~ rounds x tile width
-        const int64_t tm = (M + BM - 1) / BM;
-        const int sms = device_sm_count();
-        auto cost = [&](int bn) {
-            const int64_t tiles = tm * ((N + bn - 1) / bn);
-            return ((tiles + sms - 1) / sms) * int64_t(bn + 16);   // + per-tile fill/drain overhead
-        };
-        const int64_t c256 = cost(256), c192 = cost(192), c128 = cost(128);
-        if (c256 <= c192 && c256 <= c128) return launch<256, false, false>(a, w, M, N, K, ep, st);
-        if (c192 <= c128) return launch<192, false, false>(a, w, M, N, K, ep, st);
-        return launch<128, false, false>(a, w, M, N, K, ep, st);
-    }
-    if (ap) return launch<256, true, false>(a, w, M, N, K, ep, st);
-    return launch<256, false, true>(a, w, M, N, K, ep, st);
+    if (!ap && !wp && qgemm_tc2_supported(M, N, K, a_bits, w_bits)) return launch_qgemm_tc2(a, w, M, N, K, ep, st);
+    // Tile width by estimated time: rounds of tiles over the SMs x what one tile costs per unit of K.  Byte-lane
+    // operands cost their TMA bytes; a packed operand costs its rows again in the unpack warps, the 128 token
+    // rows in every tile, so few tokens with packed weights want narrow tiles that reach every SM.
+    const int64_t tm = (M + BM - 1) / BM;
+    const int sms = device_sm_count();
+    auto cost = [&](int bn) {
+        const int64_t tiles = tm * ((N + bn - 1) / bn);
+        return ((tiles + sms - 1) / sms) * int64_t((ap ? 2 * BM : BM / 2) + (wp ? 2 * bn : bn / 2) + 24);
+    };
+    int best = 256;
+    for (int bn : {192, 160, 128, 96, 64})
+        if (cost(bn) < cost(best)) best = bn;
+#define QLLM_TC(BN_, AP_, WP_) launch<BN_, AP_, WP_>(a, w, M, N, K, ep, st)
+#define QLLM_TC_BN(AP_, WP_) \
+    (best == 256 ? QLLM_TC(256, AP_, WP_) : best == 192 ? QLLM_TC(192, AP_, WP_) : best == 160 ? QLLM_TC(160, AP_, WP_) : \
+     best == 128 ? QLLM_TC(128, AP_, WP_) : best == 96 ? QLLM_TC(96, AP_, WP_) : QLLM_TC(64, AP_, WP_))
+    if (ap && wp) return QLLM_TC_BN(true, true);
+    if (!ap && !wp) return QLLM_TC_BN(false, false);
+    if (ap) return QLLM_TC_BN(true, false);
+    return QLLM_TC_BN(false, true);
+#undef QLLM_TC_BN
+#undef QLLM_TC
 }
 
 }  // namespace qllm

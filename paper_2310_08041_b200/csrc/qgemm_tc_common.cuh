@@ -48,11 +48,11 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, con
 // operand holds byte codes in natural order) the nibbles are interleaved back into K order.
 template <int ROWS, bool PAIRED>
 __device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ raw, uint8_t* __restrict__ op, int t) {
-    constexpr int PER_THREAD = ROWS * 4 / (32 * kUnpackWarps);
-    static_assert(PER_THREAD * 32 * kUnpackWarps == ROWS * 4, "tile rows must split evenly over the unpack threads");
+    constexpr int PER_THREAD = (ROWS * 4 + 32 * kUnpackWarps - 1) / (32 * kUnpackWarps);
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
         const int q = t + i * 32 * kUnpackWarps;
+        if (PER_THREAD * 32 * kUnpackWarps != ROWS * 4 && q >= ROWS * 4) break;   // last round of a tile that does not split evenly
         const int r = q >> 2, j = q & 3;
         const uint4 w = *reinterpret_cast<const uint4*>(raw + q * 16);
         uint4 lo, hi;
