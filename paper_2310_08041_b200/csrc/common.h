@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <utility>
 
 #include "../../include/qllm.h"
 
@@ -32,6 +33,26 @@ inline int after_launch(int n_launches = 1) {
         cudaError_t _e = (expr);                              \
         if (_e != cudaSuccess) return ::qllm::cuda_fail(_e);  \
     } while (0)
+
+// Launches kern as a programmatic dependent of the kernel launched just before it on the stream: its CTAs may
+// start once that kernel's CTAs have executed griddepcontrol.launch_dependents (or ended), and whatever it does
+// before its own griddepcontrol.wait overlaps that kernel's tail and the launch latency.  Before the wait it may
+// only touch what no earlier kernel on the stream writes or reads-then-expects-unchanged (prefetches qualify).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool bits_ok(int b) { return b == 4 || b == 6 || b == 8; }

@@ -97,8 +97,19 @@ qgemm_decode_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ w
             buf[u] = (it0 + u < iters) ? __ldcs(wp + 4 * (it0 + u)) : make_uint4(0, 0, 0, 0);
     };
 
-    // first weights are requested before the token rows are expanded: the stream starts at once
+    // The kernel is launched as a programmatic dependent of the kernel before it (the pre-GEMM kernel that writes
+    // the tokens): until that kernel is complete (griddepcontrol.wait) it only asks for its first weight rows to
+    // be brought into L2 -- harmless whoever wrote them -- so the launch latency and the first trip to HBM pass
+    // under the previous kernel.
     int task = blockIdx.x * nwarps + warp;
+    if (task < tasks) {
+        const int n_first = min(task * 8, N - 1), n_rows = min(8, N - n_first);
+        const char* base = reinterpret_cast<const char*>(w + size_t(n_first) * row_bytes);
+        for (int o = lane * 128; o < n_rows * row_bytes; o += 32 * 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(base + o));
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // first weights are requested before the token rows are expanded: the stream starts at once
     uint4 cur[UN], nxt[UN];
     const uint4* wp = nullptr;
     if (task < tasks) { wp = row_ptr(task); load_block(cur, wp, 0); }
@@ -204,7 +215,7 @@ int launch(const uint8_t* a, const uint8_t* w, int M, int N, int K, int a_bits, 
     const int sms = device_sm_count();
     const int grid = std::min(sms, tasks);
     const int wpc = tasks <= sms * 8 ? 8 : pick_warps(tasks, sms);
-    kern<<<grid, 32 * wpc, smem, st>>>(a, w, M, N, K, a_bits, ep, tasks);
+    QLLM_CUDA_TRY(launch_dependent(kern, dim3(grid), dim3(32 * wpc), smem, st, a, w, M, N, K, a_bits, ep, tasks));
     return after_launch();
 }
 

@@ -513,6 +513,8 @@ reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps
     uint2* s_lent = reinterpret_cast<uint2*>(s_lmeta + kLongRows);              // [kLongCap] their entries
     float* rows = reinterpret_cast<float*>(s_lent + kLongCap);
 
+    // a kernel launched as this one's programmatic dependent (the decode GEMM) may start its prologue now
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const int warp = __shfl_sync(0xffffffffu, int(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
     if (warp / G < TOK) {                                  // first row of this token slot towards L2
