@@ -205,3 +205,32 @@ def test_forward_under_stream_capture():
         assert torch.equal(chk, refs[rep % 2])
     for layer in layers:
         layer.destroy()
+
+
+def test_decode_calls_back_to_back_see_their_own_tokens():
+    """The decode GEMM starts its prologue while the pre-GEMM kernel of the same call still runs (a programmatic
+    dependent launch) and must wait for that kernel before it reads the tokens: forward calls issued back to back
+    with alternating inputs return, every time, the bits of the same call made alone."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    cfg = synth.CONFIGS["c3"].scaled(M=16, N=2048)
+    L = parity.oracle_layer(cfg)
+    h = B.qllm_build_reassembly(L["absmax"], L["theta"], L["W"], L["lrA"], L["lrB"], cfg.w_bits)
+    layer = B.Layer(h, L["gamma"], L["beta"], cfg.ln_eps, None, cfg.a_bits, B.QLLM_BF16, B.QLLM_BF16, max_M=cfg.M)
+    xs = [G.dev_x(synth.activations(cfg, stream=s)) for s in (1, 5, 6)]
+    refs = []
+    for x in xs:
+        ref = torch.zeros((cfg.M, cfg.N), dtype=torch.bfloat16, device=G.DEV)
+        layer.forward(x, ref)
+        torch.cuda.synchronize()
+        refs.append(ref)
+    assert not torch.equal(refs[0], refs[1])
+    outs = [torch.zeros_like(refs[0]) for _ in range(60)]
+    for i, o in enumerate(outs):                        # no synchronisation between the calls
+        layer.forward(xs[i % 3], o)
+    torch.cuda.synchronize()
+    assert B.qllm_poll_status() == 0
+    for i, o in enumerate(outs):
+        assert torch.equal(o, refs[i % 3]), i
+    layer.destroy()
