@@ -95,6 +95,10 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // The kernel is launched as a programmatic dependent of the kernel before it on the stream (for a layer, the
+    // pre-GEMM kernel that writes the tokens): everything above touched no global memory and has run under that
+    // kernel and the launch latency; nothing below starts before that kernel is complete.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -228,7 +232,7 @@ int launch(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const Ep
     QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, T::SMEM));
     const int64_t tiles = ((M + BM - 1) / BM) * int64_t((N + BN - 1) / BN);
     const int grid = int(std::min<int64_t>(tiles, device_sm_count()));
-    kern<<<grid, T::THREADS, T::SMEM, st>>>(tmA, tmW, M, N, K, ep, status);
+    QLLM_CUDA_TRY(launch_dependent(kern, dim3(grid), dim3(T::THREADS), T::SMEM, st, tmA, tmW, M, N, K, ep, status));
     return after_launch();
 }
 
