@@ -20,6 +20,9 @@ SHAPES = [
     (600, 272, 256, 4, 4), (520, 136, 512, 8, 4), (513, 80, 160, 4, 8),
     # CTA-pair kernel edges: one row past a 128-row block, narrowest output, K that ends inside a stage, 1000^3
     (129, 8, 128, 8, 8), (385, 264, 272, 8, 8), (1000, 1000, 1008, 6, 6),
+    # decode kernel edges: K that splits unevenly over a warp pair, a single 64-byte step (one warp of the pair idle),
+    # a last task with 8 of 16 channels, 9 tokens (second MMA half empty), two tasks per warp pair
+    (9, 40, 384, 4, 4), (16, 17, 128, 4, 4), (7, 2408, 640, 6, 6), (2, 24000, 128, 4, 4),
 ]
 
 
