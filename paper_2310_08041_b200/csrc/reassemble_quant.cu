@@ -804,7 +804,11 @@ int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage&
     const int sms = device_sm_count();
     const int grid = int(M < sms ? M : sms);
     const int64_t per_cta = (M + grid - 1) / grid;
-    const int tok = int(per_cta < tok_fit ? per_cta : tok_fit);
+    // the fewest rounds that the token slots allow, then the fewest slots that still make those rounds: every
+    // round is equally full on every SM (2048 tokens on 148 SMs: two rounds of 7 instead of 8 + 6 on some SMs and
+    // 8 + 0 on others), and a slot less leaves its share of shared-memory bandwidth to the others
+    const int64_t rounds = (per_cta + tok_fit - 1) / tok_fit;
+    const int tok = int((per_cta + rounds - 1) / rounds);
     int W = tok * G;
     if (W < 4) W = 4;                                       // spare warps help copy the records
     const size_t smem = size_t(fixed) + size_t(tok) * row_words * 4;
