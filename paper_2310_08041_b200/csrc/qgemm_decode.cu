@@ -123,9 +123,10 @@ qgemm_decode_kernel(const uint8_t* __restrict__ a, const uint8_t* __restrict__ w
     };
 
     // The kernel is launched as a programmatic dependent of the kernel before it (the pre-GEMM kernel that writes
-    // the tokens): until that kernel is complete (griddepcontrol.wait) it only asks for its first weight rows to
-    // be brought into L2 -- harmless whoever wrote them -- so the launch latency and the first trip to HBM pass
-    // under the previous kernel.
+    // the tokens): until that kernel is complete (griddepcontrol.wait) it only asks for the weight rows of its
+    // first task to be brought into L2 -- harmless whoever wrote them -- so the launch latency and the first trip
+    // to HBM pass under the previous kernel.  (Requesting register blocks as well before the wait delayed that
+    // kernel's own loads and made the step longer; without the L2 requests the step is 1.7 us longer.)
     int task = blockIdx.x * npairs + pair;
     if (task < tasks) {
         const int n_first = min(task * 16, N - 1), n_rows = min(16, N - n_first);
