@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libqllm_b200.so")
 
-SOURCES = ["api.cu", "builder.cpp", "reassemble_quant.cu", "reassemble_quant_generic.cu",
+SOURCES = ["api.cu", "builder.cpp", "reassemble_quant.cu", "reassemble_quant_token.cu", "reassemble_quant_generic.cu",
            "qgemm_plain.cu", "qgemm_decode.cu", "qgemm_tc.cu", "qgemm_tc2.cu", "qgemm_noalloc.cu", "theta_search.cu", "channel_distance.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

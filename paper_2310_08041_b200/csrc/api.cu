@@ -6,6 +6,7 @@
 #include <vector>
 
 #include "common.h"
+#include "reassemble_quant_common.cuh"
 
 namespace qllm {
 
@@ -222,7 +223,7 @@ struct qllm_layer {
     float *w_scale = nullptr, *w_zero = nullptr, *a_scale = nullptr, *a_zero = nullptr;
     void *x_dev = nullptr, *out_dev = nullptr;   // staging for the host-buffer entry point
     uint8_t* map_image = nullptr;                // reassembly map compiled for the fused kernel (or null)
-    int map_slots = -1;                          // its number of multi-entry rows
+    MapCounts map_counts;                        // its counts of multi-entry rows
     // The byte expansion of the 4-bit weights that a large-M GEMM needs does not depend on the tokens, so the
     // pre-GEMM call starts it on a side stream; the GEMM call joins it.
     cudaStream_t side = nullptr;
@@ -268,7 +269,7 @@ static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const 
                             const float* ln_beta, float ln_eps, const int32_t* map_ptr,
                             const int32_t* map_src, const float* map_coef, int bits, const void* map_image,
                             uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream,
-                            bool byte_lanes = false, int slots_known = -1, bool share_sm = false) {
+                            bool byte_lanes = false, const MapCounts* counts = nullptr, bool share_sm = false) {
     if (!bits_ok(bits)) return QLLM_ERR_BITS;
     if (!dtype_ok(x_dtype)) return QLLM_ERR_DTYPE;
     if (M < 0 || C <= 0 || C > 49152 || (bits == 4 && (C & 1))) return QLLM_ERR_SHAPE;
@@ -278,7 +279,7 @@ static int reassemble_entry(const void* x, int x_dtype, int64_t M, int C, const 
     if (!aligned16(x) || !aligned16(codes)) return QLLM_ERR_ALIGN;
     return launch_reassemble_quant(x, x_dtype, M, C, ln_gamma, ln_beta, ln_eps, map_ptr, map_src,
                                    map_coef, bits, map_image, codes, a_scale, a_zero, a_rowsum,
-                                   static_cast<cudaStream_t>(stream), byte_lanes, slots_known, share_sm);
+                                   static_cast<cudaStream_t>(stream), byte_lanes, counts, share_sm);
 }
 
 int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* ln_gamma,
@@ -351,11 +352,11 @@ int qllm_layer_create(const qllm_reassembly_t* h, const float* ln_gamma, const f
     step(dev_upload(L, &L->w_scale, ws, size_t(N)));
     step(dev_upload(L, &L->w_zero, wz, size_t(N)));
     step(dev_upload(L, &L->w_colsum, wcs, size_t(N)));
-    const size_t image_bytes = reassemble_map_image_bytes(C);
+    const size_t image_bytes = reassemble_map_image_bytes(C, x_dtype);
     if (image_bytes) {
         step(dev_alloc(L, &L->map_image, image_bytes));
-        if (rc == QLLM_OK) step(compile_reassemble_map(C, L->gamma, L->beta, L->ptr, L->src, L->coef, L->map_image, nullptr));
-        if (rc == QLLM_OK) step(reassemble_map_slots(C, L->map_image, nullptr, &L->map_slots));
+        if (rc == QLLM_OK) step(compile_reassemble_map(C, x_dtype, L->gamma, L->beta, L->ptr, L->src, L->coef, L->map_image, nullptr));
+        if (rc == QLLM_OK) step(reassemble_map_counts(C, x_dtype, L->map_image, nullptr, &L->map_counts));
     }
     step(dev_alloc(L, &L->codes, size_t(max_M) * size_t(C)));   // room for one code per byte
     step(dev_alloc(L, &L->a_scale, size_t(max_M)));
@@ -426,7 +427,7 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
     }
     return reassemble_entry(x, L->x_dtype, M, L->C, L->gamma, L->beta, L->eps, L->ptr, L->src, L->coef,
                             L->a_bits, L->map_image, L->codes, L->a_scale, L->a_zero, L->a_rowsum, stream,
-                            byte_lanes, L->map_image ? L->map_slots : -1, L->w_ready != nullptr);
+                            byte_lanes, L->map_image ? &L->map_counts : nullptr, L->w_ready != nullptr);
 }
 
 int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {

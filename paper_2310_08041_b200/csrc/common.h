@@ -84,26 +84,42 @@ struct EpilogueArgs {
 enum ScratchKind { kScratchExpand = 0, kScratchMapImage = 1, kScratchKinds = 2 };
 int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out);
 
-// The specialised fused kernel consumes a compiled image of the reassembly map (0 bytes: the channel
-// count has no specialised kernel).  map_image = nullptr compiles one per call into stream scratch.
-size_t reassemble_map_image_bytes(int C);
+// The specialised fused kernels consume a compiled image of the reassembly map (0 bytes: the channel
+// count has no specialised kernel; x_dtype selects the kernel: bf16 rows of 4096, 5120 or 8192 channels have
+// one of their own).  map_image = nullptr compiles one per call into stream scratch.
+struct MapCounts;
+size_t reassemble_map_image_bytes(int C, int x_dtype);
 // true when the fused kernel for C channels can write 4-bit codes one per byte (byte_lanes below)
 bool reassemble_byte_lanes_supported(int C);
-int compile_reassemble_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
-                           const float* coef, void* image, cudaStream_t st);
+int compile_reassemble_map(int C, int x_dtype, const float* gamma, const float* beta, const int32_t* ptr,
+                           const int32_t* src, const float* coef, void* image, cudaStream_t st);
+// counts: what reassemble_map_counts returned for this image (sizes the kernel's shared memory exactly instead
+// of for the largest image), or nullptr.  share_sm: another kernel of the caller runs beside this one; leave part
+// of each SM's registers to it.
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                             const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
                             float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes = false,
-                            int slots_known = -1, bool share_sm = false);
-// Counts of the multi-entry rows of a compiled image, packed into one int (waits for the stream); passing it to
-// the launcher as slots_known sizes the kernel's shared memory exactly instead of for the largest image.  share_sm: another kernel
-// of the caller runs beside this one; leave part of each SM's registers to it.
-int reassemble_map_slots(int C, const void* image, cudaStream_t st, int* slots);
+                            const MapCounts* counts = nullptr, bool share_sm = false);
+// Counts of the multi-entry rows of a compiled image (waits for the stream).
+int reassemble_map_counts(int C, int x_dtype, const void* image, cudaStream_t st, MapCounts* out);
+// The kernel for bf16 rows of LLaMA hidden sizes (reassemble_quant_token.cu)
+bool token_kernel_serves(int C);
+size_t token_image_bytes(int C);
+int compile_token_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
+                      const float* coef, void* image, cudaStream_t st);
+int token_map_counts(int C, const void* image, cudaStream_t st, MapCounts* out);
+// device word of a compiled token image: non-zero when the token kernel serves the map
+const int* token_image_served_flag(int C, const void* image);
+int launch_reassemble_quant_token(const void* x, int64_t M, int C, const float* gamma, const float* beta, float eps,
+                                  const int32_t* ptr, const int32_t* src, const float* coef, int bits,
+                                  const void* image, const MapCounts& mc, uint8_t* codes, float* a_scale,
+                                  float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes, bool share_sm);
 int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                                     const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                                     const float* coef, int bits, uint8_t* codes, float* a_scale,
-                                    float* a_zero, int32_t* a_rowsum, cudaStream_t st);
+                                    float* a_zero, int32_t* a_rowsum, cudaStream_t st,
+                                    const int* skip_if_nonzero = nullptr);
 // y[t][c] = LayerNorm(x[t])[c] in fp32 (build-time helper)
 int launch_layernorm_rows(const void* x, int x_dtype, int64_t T, int C, const float* gamma, const float* beta,
                           float eps, float* y, cudaStream_t st);

@@ -27,62 +27,16 @@
 
 #include "common.h"
 #include "device_utils.cuh"
+#include "reassemble_quant_common.cuh"
 
 namespace qllm {
 
 namespace {
 
-constexpr int kSlotCap = 2048;                 // virtual slots an image can describe
-constexpr int kInline = 4;                     // entries held inside a slot record
-constexpr int kLongCap = 512;                  // entries of longer rows kept as (position, weight) pairs
-constexpr int kLongRows = 256;                 // longer rows listed by slot (more: the slot pass scans for them)
 constexpr int kMaxWarps = 16;
-constexpr int kSmemBudget = 227 * 1024;
-constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23
-constexpr int kMagicBits = 0x4B400000;
 
 // position of channel k in a warp's row
 __host__ __device__ __forceinline__ int dplane(int k, int C) { return (k & 7) * (C >> 3) + (k >> 3); }
-
-__device__ __forceinline__ float redux_min(float v) {
-    float r;
-    asm volatile("redux.sync.min.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
-    return r;
-}
-__device__ __forceinline__ float redux_max(float v) {
-    float r;
-    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
-    return r;
-}
-__device__ __forceinline__ float min3(float a, float b, float c) {
-    float r;
-    asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
-// d = sat_u4(a) << 4 | sat_u4(b) | c << 8
-__device__ __forceinline__ uint32_t pack_sat_u4(int a, int b, uint32_t c) {
-    uint32_t d;
-    asm("cvt.pack.sat.u4.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-// d = sat_u8(a) << 8 | sat_u8(b) | c << 16
-__device__ __forceinline__ uint32_t pack_sat_u8(int a, int b, uint32_t c) {
-    uint32_t d;
-    asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(uint32_t(__cvta_generic_to_shared(smem))), "l"(gmem)
-                 : "memory");
-}
-__device__ __forceinline__ void prefetch_l2(const void* p) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
 
 // Compiled map: one allocation, in this order.
 //   idx  uint16[C]      word position in the row of the channel's (first or only) source, or C + slot
@@ -100,7 +54,6 @@ __device__ __forceinline__ void prefetch_l2(const void* p) {
 //                       than kInline (count kernel)
 // The slots serve a launch when n2 + n34 <= the row's slot room, n34 <= the room for p23/w2/w3 and all longer
 // rows are listed; otherwise the launch walks the CSR arrays.
-constexpr int kOtherCap = 1024;
 struct WarpImage {
     uint16_t* idx;
     float *wlo, *whi, *blo, *bhi;
@@ -235,13 +188,6 @@ __device__ __forceinline__ void load8<float>(const float* p, float (&f)[8]) {
     f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w;
     f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
 }
-
-struct RawMap {
-    const float* gamma;
-    const int32_t* ptr;
-    const int32_t* src;
-    const float* coef;
-};
 
 // sum_j coef_j gamma[src_j] d[pos(src_j)] over CSR entries [j0, j0 + n)
 __device__ __forceinline__ float csr_row(const RawMap& rm, const float* d, int C, int j0, int n) {
@@ -459,295 +405,6 @@ reassemble_quant_warp(const XT* __restrict__ x, int64_t M, int C, float eps, int
     }
 }
 
-// ---- compile-time channel counts ---------------------------------------------------------
-// Same algorithm with the shape fixed at compile time (LLaMA hidden sizes): G warps share a token,
-// a lane owns NPL = C / (32 G) channels, 8 consecutive ones per step.  The whole row is loaded
-// with all its 16-byte loads in flight, converted once, and the reassembled values x' stay in
-// registers between the range pass and the quantize pass, so each channel is gathered once.
-// Positions stay 16-bit and slot records are split by field (and by row length) in shared memory: what limits
-// the kernel is the number of shared-memory wavefronts per token and the tokens that fit beside the records.
-template <int G>
-__device__ __forceinline__ void token_sync(int barid) {
-    if (G == 1) __syncwarp();
-    else asm volatile("bar.sync %0, %1;" ::"r"(barid), "n"(32 * G) : "memory");
-}
-// Sum over the G warps of a token; every lane returns the total.  ex: [2][G] floats, parity-buffered.
-template <int G>
-__device__ __forceinline__ float token_sum(float v, float* ex, int& par, int wsub, int lane, int barid) {
-    v = warp_sum(v);
-    if (G == 1) { __syncwarp(); return v; }
-    if (lane == 0) ex[par * G + wsub] = v;
-    token_sync<G>(barid);
-    float t = 0.f;
-#pragma unroll
-    for (int w = 0; w < G; ++w) t += ex[par * G + w];
-    par ^= 1;
-    return t;
-}
-
-template <int NPL, int G, bool HAS_BETA, bool PACKED, int MAXW>
-__global__ void __launch_bounds__(32 * MAXW, 1)
-reassemble_quant_token(const __nv_bfloat16* __restrict__ x, int64_t M, float eps, int bits, WarpImage im,
-                       int row_words, int other_room, int TOK /* tokens in flight per CTA */, RawMap rm,
-                       uint8_t* __restrict__ codes, float* __restrict__ a_scale,
-                       float* __restrict__ a_zero, int32_t* __restrict__ a_rowsum) {
-    constexpr int C = NPL * 32 * G;
-    constexpr int NIT = NPL / 8;                           // steps of 8 channels per lane
-    constexpr int P = C / 8;                               // plane stride in words
-    constexpr int GS = 32 * G;                             // groups per step over the token's lanes
-    extern __shared__ __align__(16) uint8_t smem_bytes[];
-    float* s_wA = reinterpret_cast<float*>(smem_bytes);    // [C/8][4] weights of channels 8g..8g+3
-    float* s_wB = s_wA + C / 2;                            //                      channels 8g+4..8g+7
-    float* s_bA = s_wB + C / 2;                            // bias arrays only with beta
-    float* s_bB = s_bA + C / 2;
-    uint16_t* s_idx = reinterpret_cast<uint16_t*>(HAS_BETA ? s_bB + C / 2 : s_bA);     // [C] word positions
-    float* s_ex = reinterpret_cast<float*>(s_idx + C);                  // [MAXW / G][8 G] exchange words per token slot
-    const int slot_room = row_words - C;
-    uint32_t* s_p01 = reinterpret_cast<uint32_t*>(s_ex + (MAXW / G) * 8 * G);   // slot records, field by field
-    float* s_w0 = reinterpret_cast<float*>(s_p01 + slot_room);
-    float* s_w1 = s_w0 + slot_room;
-    uint32_t* s_p23 = reinterpret_cast<uint32_t*>(s_w1 + slot_room);
-    float* s_w2 = reinterpret_cast<float*>(s_p23 + other_room);
-    float* s_w3 = s_w2 + other_room;
-    int4* s_lmeta = reinterpret_cast<int4*>(s_w3 + other_room);                 // [kLongRows] rows longer than a record
-    uint2* s_lent = reinterpret_cast<uint2*>(s_lmeta + kLongRows);              // [kLongCap] their entries
-    float* rows = reinterpret_cast<float*>(s_lent + kLongCap);
-
-    // a kernel launched as this one's programmatic dependent (the decode GEMM) may start its prologue now
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int lane = threadIdx.x & 31;
-    const int warp = __shfl_sync(0xffffffffu, int(threadIdx.x >> 5), 0);   // warp-uniform for the compiler
-    if (warp / G < TOK) {                                  // first row of this token slot towards L2
-        const int64_t m0 = int64_t(blockIdx.x) * TOK + warp / G;
-        if (m0 < M) {
-            const char* x0 = reinterpret_cast<const char*>(x + m0 * C);
-            for (int o = ((warp % G) * 32 + lane) * 128; o < C * 2; o += GS * 128) prefetch_l2(x0 + o);
-        }
-    }
-    {   // records -> shared memory, asynchronously: they are first needed after the first row's statistics
-        const uint4* gw = reinterpret_cast<const uint4*>(im.wlo);       // wlo | whi | blo | bhi back to back
-        const int nw16 = (HAS_BETA ? 8 : 4) * C / 16;
-        for (int i = threadIdx.x; i < nw16; i += blockDim.x) cp_async16(reinterpret_cast<uint4*>(s_wA) + i, gw + i);
-        auto copy16 = [&](void* dst, const void* src, int n16) {
-            for (int i = threadIdx.x; i < n16; i += blockDim.x)
-                cp_async16(static_cast<uint4*>(dst) + i, static_cast<const uint4*>(src) + i);
-        };
-        copy16(s_idx, im.idx, 2 * C / 16);
-        copy16(s_p01, im.p01, slot_room / 4);
-        copy16(s_w0, im.w0, slot_room / 4);
-        copy16(s_w1, im.w1, slot_room / 4);
-        copy16(s_p23, im.p23, other_room / 4);
-        copy16(s_w2, im.w2, other_room / 4);
-        copy16(s_w3, im.w3, other_room / 4);
-        copy16(s_lmeta, im.lmeta, kLongRows);
-        copy16(s_lent, im.lent, kLongCap / 2);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-    }
-    const bool slow = !slots_fit(im.head, slot_room, other_room);   // uniform over the grid: walk the CSR arrays
-    const int n2 = slow ? 0 : __ldg(im.head + 4);          // slots of two-entry rows come first
-    const int nslots = slow ? 0 : n2 + __ldg(im.head + 5);
-    const int nlong = slow ? 0 : __ldg(im.head + 6);       // rows longer than a slot record
-    bool records_pending = true;
-
-    const int tslot = warp / G, wsub = warp % G;
-    if (tslot >= TOK) {                                    // spare warps only helped with the copy
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncthreads();
-        return;
-    }
-    const int barid = 1 + tslot;
-    float* d = rows + size_t(tslot) * row_words;
-    float* ex = s_ex + tslot * 8 * G;
-    float* exr = ex + 2 * G;                               // range exchange: [2][G][2]
-    const int g0 = wsub * 32 + lane;                       // this lane's group in step 0
-    const float invC = 1.0f / float(C);
-    const float qmax = float((1 << bits) - 1);
-    const float inv_qmax = 1.0f / qmax;
-    const int top = int(qmax);
-    const int64_t stride = int64_t(gridDim.x) * TOK;
-    int par = 0;
-
-    for (int64_t m = int64_t(blockIdx.x) * TOK + tslot; m < M; m += stride) {
-        const __nv_bfloat16* xr = x + m * C + 8 * g0;
-        uint4 raw[NIT];
-#pragma unroll
-        for (int i = 0; i < NIT; ++i) raw[i] = *reinterpret_cast<const uint4*>(xr + i * 8 * GS);
-        // -- mean
-        float s = 0.f;
-#pragma unroll
-        for (int i = 0; i < NIT; ++i) {
-            const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-            float t = 0.f;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) t += __uint_as_float(w[k] << 16) + __uint_as_float(w[k] & 0xFFFF0000u);
-            s += t;
-        }
-        const float mean = token_sum<G>(s, ex, par, wsub, lane, barid) * invC;
-        // -- centred row to the token's planes, variance
-        float sq = 0.f;
-#pragma unroll
-        for (int i = 0; i < NIT; ++i) {
-            const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float a = __uint_as_float(w[k] << 16) - mean;
-                const float b = __uint_as_float(w[k] & 0xFFFF0000u) - mean;
-                sq = fmaf(a, a, sq);
-                sq = fmaf(b, b, sq);
-                d[(2 * k) * P + g0 + i * GS] = a;
-                d[(2 * k + 1) * P + g0 + i * GS] = b;
-            }
-        }
-        // the exchange inside token_sum also makes the row visible to the token's lanes
-        const float rstd = rsqrtf(token_sum<G>(sq, ex, par, wsub, lane, barid) * invC + eps);
-        if (m + stride < M) {                              // next row of this token slot towards L2
-            const char* xn = reinterpret_cast<const char*>(x + (m + stride) * C);
-#pragma unroll
-            for (int o = 0; o < C * 2; o += GS * 128)
-                if (o + g0 * 128 < C * 2) prefetch_l2(xn + o + g0 * 128);
-        }
-        if (records_pending) {                             // first token of this warp: the records have landed
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            __syncthreads();
-            records_pending = false;
-        }
-        // -- merged rows: a lane per row sums the entries into the row's virtual slot
-        if (nslots > 0) {
-            // two-entry rows first, then the rows with entries 2 and 3 (only the warp step that straddles n2 diverges);
-            // a longer row's record carries zero weights and is patched afterwards
-#pragma unroll 4
-            for (int vi = g0; vi < nslots; vi += GS) {
-                const uint32_t p = s_p01[vi];
-                float e = s_w0[vi] * d[p & 0xFFFFu];
-                e = fmaf(s_w1[vi], d[p >> 16], e);
-                if (vi >= n2) {
-                    const uint32_t q = s_p23[vi - n2];
-                    e = fmaf(s_w2[vi - n2], d[q & 0xFFFFu], e);
-                    e = fmaf(s_w3[vi - n2], d[q >> 16], e);
-                }
-                d[C + vi] = e;
-            }
-            if (nlong > 0) token_sync<G>(barid);           // another lane wrote this slot's record value just above
-            for (int k = g0; k < nlong; k += GS) {         // few rows
-                const int4 lm = s_lmeta[k];
-                d[C + lm.x] = lm.w ? pair_row(s_lent, d, lm.y, lm.z) : csr_row(rm, d, C, lm.y, lm.z);
-            }
-            token_sync<G>(barid);
-        }
-        // -- reassembly: one gather per channel; row range
-        float v[NPL];
-        float lo = INFINITY, hi = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < NIT; ++i) {
-            const int g = g0 + i * GS;
-            const uint4 iw = reinterpret_cast<const uint4*>(s_idx)[g];     // 8 word positions
-            const float4 wa = reinterpret_cast<const float4*>(s_wA)[g], wb = reinterpret_cast<const float4*>(s_wB)[g];
-            float* u = v + 8 * i;
-            if (slow) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) u[j] = csr_channel(rm, d, C, 8 * g + j);
-            } else {
-            u[0] = wa.x * d[iw.x & 0xFFFFu]; u[1] = wa.y * d[iw.x >> 16];
-            u[2] = wa.z * d[iw.y & 0xFFFFu]; u[3] = wa.w * d[iw.y >> 16];
-            u[4] = wb.x * d[iw.z & 0xFFFFu]; u[5] = wb.y * d[iw.z >> 16];
-            u[6] = wb.z * d[iw.w & 0xFFFFu]; u[7] = wb.w * d[iw.w >> 16];
-            }
-            if (HAS_BETA) {
-                const float4 ba = reinterpret_cast<const float4*>(s_bA)[g], bb = reinterpret_cast<const float4*>(s_bB)[g];
-                u[0] = fmaf(rstd, u[0], ba.x); u[1] = fmaf(rstd, u[1], ba.y);
-                u[2] = fmaf(rstd, u[2], ba.z); u[3] = fmaf(rstd, u[3], ba.w);
-                u[4] = fmaf(rstd, u[4], bb.x); u[5] = fmaf(rstd, u[5], bb.y);
-                u[6] = fmaf(rstd, u[6], bb.z); u[7] = fmaf(rstd, u[7], bb.w);
-            }
-#pragma unroll
-            for (int j = 0; j < 8; j += 2) {
-                lo = min3(lo, u[j], u[j + 1]);
-                hi = max3(hi, u[j], u[j + 1]);
-            }
-        }
-        if (!HAS_BETA) { lo *= rstd; hi *= rstd; }         // rstd > 0: scaling commutes with min / max
-        lo = redux_min(lo);
-        hi = redux_max(hi);
-        if (G > 1) {
-            if (lane == 0) { exr[par * 2 * G + 2 * wsub] = lo; exr[par * 2 * G + 2 * wsub + 1] = hi; }
-            token_sync<G>(barid);
-#pragma unroll
-            for (int w = 0; w < G; ++w) {
-                lo = fminf(lo, exr[par * 2 * G + 2 * w]);
-                hi = fmaxf(hi, exr[par * 2 * G + 2 * w + 1]);
-            }
-        }
-        // -- Eq. 2
-        float alpha = (hi - lo) * inv_qmax;
-        if (!(hi > lo)) alpha = lo != 0.f ? fabsf(lo) : 1.f;
-        const float inv = __frcp_rn(alpha);
-        const float zero = -rintf(lo * inv);
-        const bool big = fmaxf(fabsf(lo), fabsf(hi)) * inv >= 2097152.f || fabsf(zero) >= 2097152.f;
-        const int zadd = int(zero) - kMagicBits;
-        const float sc = HAS_BETA ? inv : rstd * inv;      // without beta v holds x' / rstd
-        int csum = 0;
-#pragma unroll
-        for (int i = 0; i < NIT; ++i) {
-            const int g = g0 + i * GS;
-            const float* u = v + 8 * i;
-            int n[8];
-            if (!big) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) n[j] = __float_as_int(fmaf(u[j], sc, kMagic)) + zadd;
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) n[j] = int(fminf(fmaxf(rintf(u[j] * sc) + zero, 0.f), qmax));
-            }
-            if (PACKED) {
-                uint32_t p = 0;
-#pragma unroll
-                for (int k = 3; k >= 0; --k) p = pack_sat_u4(n[2 * k + 1], n[2 * k], p);
-                const uint32_t nib = (p & 0x0F0F0F0Fu) + ((p >> 4) & 0x0F0F0F0Fu);
-                csum = int(__dp4a(nib, 0x01010101u, uint32_t(csum)));
-                *reinterpret_cast<uint32_t*>(codes + m * (C / 2) + 4 * g) = p;
-            } else {
-                uint32_t p0 = pack_sat_u8(min(n[3], top), min(n[2], top), 0u);
-                p0 = pack_sat_u8(min(n[1], top), min(n[0], top), p0);
-                uint32_t p1 = pack_sat_u8(min(n[7], top), min(n[6], top), 0u);
-                p1 = pack_sat_u8(min(n[5], top), min(n[4], top), p1);
-                csum = int(__dp4a(p0, 0x01010101u, uint32_t(csum)));
-                csum = int(__dp4a(p1, 0x01010101u, uint32_t(csum)));
-                *reinterpret_cast<uint2*>(codes + m * C + 8 * g) = make_uint2(p0, p1);
-            }
-        }
-        csum = __reduce_add_sync(0xffffffffu, csum);
-        if (G == 1) {
-            if (lane == 0) {
-                a_scale[m] = alpha;
-                a_zero[m] = zero;
-                if (a_rowsum) a_rowsum[m] = csum;
-            }
-            __syncwarp();
-        } else {
-            // partial code sums meet in the parity slot that the range exchange just used; the next
-            // token's first exchange uses the other parity, and its barrier orders these reads before
-            // any later write of this slot
-            int* exi = reinterpret_cast<int*>(exr + par * 2 * G);
-            token_sync<G>(barid);                          // everyone has read the range
-            if (lane == 0) exi[wsub] = csum;
-            token_sync<G>(barid);
-            if (wsub == 0 && lane == 0) {
-                int tot = 0;
-#pragma unroll
-                for (int w = 0; w < G; ++w) tot += exi[w];
-                a_scale[m] = alpha;
-                a_zero[m] = zero;
-                if (a_rowsum) a_rowsum[m] = tot;
-            }
-            par ^= 1;                                      // min/max exchange used parity `par`
-        }
-    }
-    if (records_pending) {                                 // a warp without tokens still joins the CTA barrier
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncthreads();
-    }
-}
-
 // warps per CTA that fit with the given slot room (0: does not fit)
 int warps_that_fit(int C, bool has_beta, int slot_room) {
     const int64_t rec = int64_t(has_beta ? 10 : 6) * C;
@@ -775,93 +432,28 @@ int launch_warp(const void* x, int64_t M, int C, float eps, int bits, const Warp
 }
 
 
-template <int NPL, int G, bool HAS_BETA, bool PACKED, int MAXW>
-int launch_token(const void* x, int64_t M, float eps, int bits, const WarpImage& im, int slot_room, int other_room,
-                 const RawMap& rm,
-                 uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool share_sm) {
-    constexpr int C = NPL * 32 * G;
-    auto kern = reassemble_quant_token<NPL, G, HAS_BETA, PACKED, MAXW>;
-    const int row_words = C + slot_room;
-    // weights (+ bias), positions, exchange words, slot records field by field, longer rows
-    const int64_t fixed = int64_t(HAS_BETA ? 8 : 4) * C + 2 * C + (MAXW / G) * 8 * G * 4 + int64_t(slot_room) * 12 +
-                          int64_t(other_room) * 12 + kLongRows * 16 + kLongCap * 8;
-    int tok_fit = int((kSmemBudget - fixed) / (int64_t(row_words) * 4));
-    if (tok_fit > MAXW / G) tok_fit = MAXW / G;
-    if (share_sm) {
-        // leave a fifth of the register file free: the layer expands its 4-bit weights for the coming GEMM
-        // on a second stream meanwhile, and that bandwidth-bound kernel needs room on every SM to keep
-        // enough loads in flight (this kernel is latency-bound and does not miss the token slot)
-        static int regs = 0;
-        if (regs == 0) {
-            cudaFuncAttributes fa;
-            QLLM_CUDA_TRY(cudaFuncGetAttributes(&fa, kern));
-            regs = fa.numRegs > 0 ? fa.numRegs : 128;
-        }
-        const int w_cap = int(0.8 * 65536 / (regs * 32));
-        if (tok_fit > w_cap / G && w_cap / G >= 1) tok_fit = w_cap / G;
-    }
-    if (tok_fit < 1) return QLLM_ERR_UNSUPPORTED;
-    const int sms = device_sm_count();
-    const int grid = int(M < sms ? M : sms);
-    const int64_t per_cta = (M + grid - 1) / grid;
-    // the fewest rounds that the token slots allow, then the fewest slots that still make those rounds: every
-    // round is equally full on every SM (2048 tokens on 148 SMs: two rounds of 7 instead of 8 + 6 on some SMs and
-    // 8 + 0 on others), and a slot less leaves its share of shared-memory bandwidth to the others
-    const int64_t rounds = (per_cta + tok_fit - 1) / tok_fit;
-    const int tok = int((per_cta + rounds - 1) / rounds);
-    int W = tok * G;
-    if (W < 4) W = 4;                                       // spare warps help copy the records
-    const size_t smem = size_t(fixed) + size_t(tok) * row_words * 4;
-    QLLM_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-    kern<<<grid, 32 * W, smem, st>>>(static_cast<const __nv_bfloat16*>(x), M, eps, bits, im, row_words, other_room, tok, rm,
-                                     codes, a_scale, a_zero, a_rowsum);
-    return after_launch();
-}
-
-// Channels per lane, warps per token, most warps per CTA of the compile-time shapes (measured best).
-#ifndef QLLM_RQ_4096
-#define QLLM_RQ_4096 64
-#define QLLM_RQ_4096_G 2
-#define QLLM_RQ_4096_W 20
-#endif
-#ifndef QLLM_RQ_5120
-#define QLLM_RQ_5120 80
-#define QLLM_RQ_5120_G 2
-#define QLLM_RQ_5120_W 16
-#endif
-#ifndef QLLM_RQ_8192
-#define QLLM_RQ_8192 64
-#define QLLM_RQ_8192_G 4
-#define QLLM_RQ_8192_W 16
-#endif
-
-template <int NPL, int G, int MAXW>
-int launch_token_variant(bool has_beta, bool packed, const void* x, int64_t M, float eps, int bits,
-                         const WarpImage& im, int slot_room, int other_room, const RawMap& rm, uint8_t* codes,
-                         float* a_scale,
-                         float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool share_sm) {
-#define QLLM_RQT(B, P) launch_token<NPL, G, B, P, MAXW>(x, M, eps, bits, im, slot_room, other_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm)
-    if (has_beta) return packed ? QLLM_RQT(true, true) : QLLM_RQT(true, false);
-    return packed ? QLLM_RQT(false, true) : QLLM_RQT(false, false);
-#undef QLLM_RQT
-}
-
 }  // namespace
 
 // ---- host entry points -----------------------------------------------------------------------
 // The warp kernel serves a channel count when the records (with bias terms) and at least one row with
-// the full slot allowance fit into shared memory; other shapes take the shape-agnostic kernel.
+// the full slot allowance fit into shared memory; other shapes take the shape-agnostic kernel.  bf16 rows
+// of the LLaMA hidden sizes take the token kernel (reassemble_quant_token.cu), which has its own image.
 static bool warp_kernel_serves(int C) {
     return C % 256 == 0 && C + kSlotCap <= 65535 && warps_that_fit(C, true, kSlotCap) >= 1;
 }
+static bool token_path(int C, int x_dtype) { return x_dtype == QLLM_BF16 && token_kernel_serves(C); }
 
 bool reassemble_byte_lanes_supported(int C) { return warp_kernel_serves(C); }
 
-size_t reassemble_map_image_bytes(int C) { return warp_kernel_serves(C) ? warp_image_bytes(C) : 0; }
+// Token path: the image is the token kernel's, followed by the warp kernel's (used when the token kernel cannot
+// serve the map: slots beyond its limits, or source channels read by several rows with different coefficients).
+size_t reassemble_map_image_bytes(int C, int x_dtype) {
+    if (token_path(C, x_dtype)) return token_image_bytes(C) + warp_image_bytes(C);
+    return warp_kernel_serves(C) ? warp_image_bytes(C) : 0;
+}
 
-int compile_reassemble_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
-                           const float* coef, void* image, cudaStream_t st) {
-    if (!warp_kernel_serves(C)) return QLLM_ERR_UNSUPPORTED;
+static int compile_warp_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
+                            const float* coef, void* image, cudaStream_t st) {
     const WarpImage im = warp_image_at(image, C);
     QLLM_CUDA_TRY(cudaMemsetAsync(im.head, 0, 32, st));
     count_rows_kernel<<<(C + 255) / 256, 256, 0, st>>>(C, ptr, im);
@@ -869,63 +461,85 @@ int compile_reassemble_map(int C, const float* gamma, const float* beta, const i
     return after_launch(2);
 }
 
-int reassemble_map_slots(int C, const void* image, cudaStream_t st, int* slots) {
+int compile_reassemble_map(int C, int x_dtype, const float* gamma, const float* beta, const int32_t* ptr,
+                           const int32_t* src, const float* coef, void* image, cudaStream_t st) {
+    if (token_path(C, x_dtype)) {
+        const int rc = compile_token_map(C, gamma, beta, ptr, src, coef, image, st);
+        if (rc != QLLM_OK) return rc;
+        return compile_warp_map(C, gamma, beta, ptr, src, coef, static_cast<uint8_t*>(image) + token_image_bytes(C), st);
+    }
+    if (!warp_kernel_serves(C)) return QLLM_ERR_UNSUPPORTED;
+    return compile_warp_map(C, gamma, beta, ptr, src, coef, image, st);
+}
+
+int reassemble_map_counts(int C, int x_dtype, const void* image, cudaStream_t st, MapCounts* out) {
+    if (token_path(C, x_dtype)) return token_map_counts(C, image, st, out);
     if (!warp_kernel_serves(C)) return QLLM_ERR_UNSUPPORTED;
     const WarpImage im = warp_image_at(const_cast<void*>(image), C);
     int head[8];
     QLLM_CUDA_TRY(cudaMemcpyAsync(head, im.head, sizeof(head), cudaMemcpyDeviceToHost, st));
     QLLM_CUDA_TRY(cudaStreamSynchronize(st));
-    // rows with two entries + rows with more, and the latter again in the upper half; -1 (unknown: the launcher
-    // then assumes the largest image) when the image's slots cannot serve a launch anyway
-    const bool fits = head[4] + head[5] <= kSlotCap && head[5] <= kOtherCap && head[6] <= kLongRows;
-    *slots = fits ? ((head[5] << 16) | (head[4] + head[5])) : -1;
+    MapCounts mc;
+    mc.known = true;
+    mc.slots = head[4] + head[5];
+    mc.other = head[5];
+    mc.long_rows = head[6];
+    mc.long_entries = head[1] <= kLongCap ? head[1] : kLongCap;
+    mc.fits = mc.slots <= kSlotCap && mc.other <= kOtherCap && mc.long_rows <= kLongRows;
+    *out = mc;
     return QLLM_OK;
 }
 
 int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                             const float* beta, float eps, const int32_t* ptr, const int32_t* src,
                             const float* coef, int bits, const void* map_image, uint8_t* codes, float* a_scale,
-                            float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes, int slots_known,
+                            float* a_zero, int32_t* a_rowsum, cudaStream_t st, bool byte_lanes, const MapCounts* counts,
                             bool share_sm) {
     if (!warp_kernel_serves(C) || !gamma) {              // no LayerNorm: the shape-agnostic kernel
         if (byte_lanes && bits == 4) return QLLM_ERR_UNSUPPORTED;
         return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
                                                a_scale, a_zero, a_rowsum, st);
     }
+    MapCounts mc;                                          // unknown unless the caller compiled the image before
+    if (map_image && counts) mc = *counts;
+    if (token_path(C, x_dtype)) {
+        if (!map_image) {
+            // direct call: the map is compiled for this launch into per-stream library scratch (one launch); the
+            // token kernel serves it if the image says it can, else the shape-agnostic kernel behind it does
+            uint8_t* buf = nullptr;
+            int rc = stream_scratch(kScratchMapImage, st, token_image_bytes(C), &buf);
+            if (rc != QLLM_OK) return rc;
+            rc = compile_token_map(C, gamma, beta, ptr, src, coef, buf, st);
+            if (rc != QLLM_OK) return rc;
+            rc = launch_reassemble_quant_token(x, M, C, gamma, beta, eps, ptr, src, coef, bits, buf, MapCounts(), codes,
+                                               a_scale, a_zero, a_rowsum, st, false, share_sm);
+            if (rc != QLLM_OK) return rc;
+            return launch_reassemble_quant_generic(x, x_dtype, M, C, gamma, beta, eps, ptr, src, coef, bits, codes,
+                                                   a_scale, a_zero, a_rowsum, st, token_image_served_flag(C, buf));
+        }
+        if (mc.known && mc.fits)
+            return launch_reassemble_quant_token(x, M, C, gamma, beta, eps, ptr, src, coef, bits, map_image, mc, codes,
+                                                 a_scale, a_zero, a_rowsum, st, byte_lanes, share_sm);
+        // the token kernel cannot serve this map: the warp kernel with its own image (counts not read back)
+        map_image = static_cast<const uint8_t*>(map_image) + token_image_bytes(C);
+        mc = MapCounts();
+    }
     if (!map_image) {
         // direct call: compile the map for this launch into per-stream library scratch
         uint8_t* buf = nullptr;
         int rc = stream_scratch(kScratchMapImage, st, warp_image_bytes(C), &buf);
         if (rc != QLLM_OK) return rc;
-        rc = compile_reassemble_map(C, gamma, beta, ptr, src, coef, buf, st);
+        rc = compile_warp_map(C, gamma, beta, ptr, src, coef, buf, st);
         if (rc != QLLM_OK) return rc;
         map_image = buf;
-        slots_known = -1;
     }
     const WarpImage im = warp_image_at(const_cast<void*>(map_image), C);
     // room for slot records and slot values: exact when the caller knows the image's counts, else the largest
-    // image's total with a quarter of it for rows of three and more entries (an image beyond the room makes the
-    // launch walk the CSR arrays)
-    int slot_room = kSlotCap, other_room = kSlotCap / 4;
-    if (slots_known >= 0) {
-        slot_room = ((slots_known & 0xFFFF) + 3) & ~3;
-        other_room = ((slots_known >> 16) + 3) & ~3;
-    }
+    // image's total (an image beyond the room makes the launch walk the CSR arrays)
+    int slot_room = kSlotCap;
+    if (mc.known && mc.fits) slot_room = (mc.slots + 3) & ~3;
     const RawMap rm{gamma, ptr, src, coef};
     const bool packed = bits == 4 && !byte_lanes, has_beta = beta != nullptr;
-    if (x_dtype == QLLM_BF16) {
-        // LLaMA hidden sizes: shape fixed at compile time
-#define QLLM_TOKEN_ARGS has_beta, packed, x, M, eps, bits, im, slot_room, other_room, rm, codes, a_scale, a_zero, a_rowsum, st, share_sm
-        if (M <= device_sm_count()) {                          // one token per CTA: spread it over more warps
-            if (C == 4096) return launch_token_variant<16, 8, 8>(QLLM_TOKEN_ARGS);
-            if (C == 5120) return launch_token_variant<40, 4, 4>(QLLM_TOKEN_ARGS);
-            if (C == 8192) return launch_token_variant<16, 16, 16>(QLLM_TOKEN_ARGS);
-        }
-        if (C == 4096) return launch_token_variant<QLLM_RQ_4096, QLLM_RQ_4096_G, QLLM_RQ_4096_W>(QLLM_TOKEN_ARGS);
-        if (C == 5120) return launch_token_variant<QLLM_RQ_5120, QLLM_RQ_5120_G, QLLM_RQ_5120_W>(QLLM_TOKEN_ARGS);
-        if (C == 8192) return launch_token_variant<QLLM_RQ_8192, QLLM_RQ_8192_G, QLLM_RQ_8192_W>(QLLM_TOKEN_ARGS);
-#undef QLLM_TOKEN_ARGS
-    }
 #define QLLM_RQW(XT, B, P) launch_warp<XT, B, P>(x, M, C, eps, bits, im, slot_room, rm, codes, a_scale, a_zero, a_rowsum, st)
     if (x_dtype == QLLM_BF16) {
         if (has_beta) return packed ? QLLM_RQW(__nv_bfloat16, true, true) : QLLM_RQW(__nv_bfloat16, true, false);

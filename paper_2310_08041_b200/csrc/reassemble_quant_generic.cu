@@ -73,9 +73,12 @@ reassemble_quant_generic(const XT* __restrict__ x, int64_t M, int C, const float
                          const float* __restrict__ beta, float eps, const int32_t* __restrict__ ptr,
                          const int32_t* __restrict__ src, const float* __restrict__ coef, int bits,
                          uint8_t* __restrict__ codes, float* __restrict__ a_scale,
-                         float* __restrict__ a_zero, int32_t* __restrict__ a_rowsum) {
+                         float* __restrict__ a_zero, int32_t* __restrict__ a_rowsum,
+                         const int* __restrict__ skip_if_nonzero) {
     extern __shared__ float y[];
     __shared__ float red[2 * 32];
+    // launched behind a specialised kernel that may have served the call already (it says so in this word)
+    if (skip_if_nonzero && *skip_if_nonzero != 0) return;
     const float qmax = float((1 << bits) - 1);
     for (int64_t m = blockIdx.x; m < M; m += gridDim.x) {
         layernorm_row<XT>(x + m * C, C, gamma, beta, eps, y, red);
@@ -144,7 +147,8 @@ calib_absmax_kernel(const XT* __restrict__ x, int64_t M, int C, const float* __r
 int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                                     const float* beta, float eps, const int32_t* ptr,
                                     const int32_t* src, const float* coef, int bits, uint8_t* codes,
-                                    float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st) {
+                                    float* a_scale, float* a_zero, int32_t* a_rowsum, cudaStream_t st,
+                                    const int* skip_if_nonzero) {
     const size_t smem = size_t(C) * sizeof(float);
     if (smem > 200 * 1024) return QLLM_ERR_UNSUPPORTED;
     const int grid = int(std::min<int64_t>(M, int64_t(device_sm_count()) * 4));
@@ -152,12 +156,12 @@ int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C
         auto k = reassemble_quant_generic<float>;
         if (smem > 48 * 1024) QLLM_CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
         k<<<grid, kThreads, smem, st>>>(static_cast<const float*>(x), M, C, gamma, beta, eps, ptr, src,
-                                        coef, bits, codes, a_scale, a_zero, a_rowsum);
+                                        coef, bits, codes, a_scale, a_zero, a_rowsum, skip_if_nonzero);
     } else {
         auto k = reassemble_quant_generic<__nv_bfloat16>;
         if (smem > 48 * 1024) QLLM_CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)));
         k<<<grid, kThreads, smem, st>>>(static_cast<const __nv_bfloat16*>(x), M, C, gamma, beta, eps,
-                                        ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum);
+                                        ptr, src, coef, bits, codes, a_scale, a_zero, a_rowsum, skip_if_nonzero);
     }
     return after_launch();
 }

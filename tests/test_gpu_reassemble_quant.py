@@ -178,3 +178,36 @@ def test_full_size_launches_repeat_bit_for_bit(name):
         assert np.array_equal(got["stored"], first["stored"])
         assert np.array_equal(got["scale"], first["scale"]) and np.array_equal(got["zero"], first["zero"])
         assert np.array_equal(got["rowsum"], first["rowsum"])
+
+
+@pytest.mark.parametrize("kind", ["shared_sources", "unread_sources", "long_rows", "identity"])
+@pytest.mark.parametrize("C", [4096, 5120])
+def test_handmade_maps_on_the_token_kernel_shapes(kind, C):
+    """bf16 rows of a LLaMA hidden size take the kernel that works on the source side of the map.  It serves a map
+    only when every source channel is read by single-entry rows of one coefficient or by exactly one multi-entry
+    row; any other map must still give the oracle's result (the shape-agnostic kernel takes the call)."""
+    import gpu_util as G
+    rng = np.random.default_rng(17)
+    M = 37
+    x = synth.f32_to_bf16_bits((rng.standard_normal((M, C)) * (1 + 30 * (rng.random(C) < 0.01))).astype(np.float32))
+    g = (1 + 0.1 * rng.standard_normal(C)).astype(np.float32)
+    rows = []
+    for c in range(C):
+        if kind == "identity":
+            rows.append([(c, 1.0)])
+        elif kind == "shared_sources":                   # every source is read by two rows, with two coefficients
+            rows.append([(c, 0.5), ((c * 7 + 3) % C, 0.25)])
+        elif kind == "unread_sources":                   # odd sources are read by nobody, even ones by two rows (T = 2)
+            rows.append([(c & ~1, 0.5)])
+        else:                                            # rows of 1, 3 and 11 entries (longer than a slot record) that this kernel serves
+            k = c % 16
+            rows.append([(c, 1.0)] if k < 2 else ([(c - c % 16 + 2 + e, 1.0 / 3) for e in range(3)] if k == 2 else
+                        ([(c - c % 16 + 5 + e, 1.0 / 11) for e in range(11)] if k == 3 else [(c - c % 16 + (k & 1), 1.0)])))
+    ptr = np.zeros(C + 1, np.int32)
+    ptr[1:] = np.cumsum([len(r) for r in rows])
+    src = np.array([sj for r in rows for sj, _ in r], np.int32)
+    coef = np.array([cj for r in rows for _, cj in r], np.float32)
+    for bits in (4, 6):
+        got = G.run_reassemble_quant(x, g, None, 1e-5, ptr, src, coef, bits)
+        ref = oracle.reassemble_quant(x, g, None, 1e-5, ptr, src, coef, bits, want_pre=True)
+        parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref, bits)
