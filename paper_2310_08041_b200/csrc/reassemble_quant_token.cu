@@ -773,7 +773,7 @@ int launch_reassemble_quant_token(const void* x, int64_t M, int C, const float* 
     }
     if (C == 4096) return launch_token_variant<4096, 4, 20>(QLLM_TOKEN_ARGS);
     if (C == 5120) return launch_token_variant<5120, 5, 20>(QLLM_TOKEN_ARGS);
-    if (C == 8192) return launch_token_variant<8192, 8, 16>(QLLM_TOKEN_ARGS);
+    if (C == 8192) return launch_token_variant<8192, 8, 24>(QLLM_TOKEN_ARGS);
 #undef QLLM_TOKEN_ARGS
     return QLLM_ERR_UNSUPPORTED;
 }
