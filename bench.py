@@ -10,8 +10,12 @@ epilogue.  Prints ONE JSON line (rank 0).  `--impl reference` times the CPU orac
 from __future__ import annotations
 
 import argparse
+import glob
+import hashlib
 import json
+import math
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -24,9 +28,33 @@ if ROOT not in sys.path:
 
 METRIC = "W4A4 reassembled-linear tokens/s; TOPS & GB/s as % of B200 roofline"
 UNIT = "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the GEMM kernel, from the ncu captures summarised
-# under profiles/ (keyed by workload and tokens per GPU; absent = not captured for the current kernel)
-NCU_TRAFFIC = {("c2", 2048): 79.2e6, ("c3", 16): 45.4e6}
+NOMINAL_HBM_GBS = 8000.0
+
+
+def _traffic(kernel, workload, M):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `kernel`, from the ncu summaries under
+    profiles/: a line `traffic-record: kernel=.. workload=.. M=.. bytes=.. sources=a.cu,b.cuh sha256=..` holds the
+    counter and the hash of the kernel's sources when it was taken.  None when there is no record for this
+    workload or the sources have changed since (the counter is then stale)."""
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        for line in open(path):
+            if not line.startswith("traffic-record:"):
+                continue
+            kv = dict(tok.split("=", 1) for tok in line.split()[1:] if "=" in tok)
+            if kv.get("kernel") != kernel or kv.get("workload") != workload or int(kv.get("M", -1)) != M:
+                continue
+            h = hashlib.sha256()
+            for src in kv.get("sources", "").split(","):
+                f = os.path.join(ROOT, "paper_2310_08041_b200", "csrc", src)
+                if not os.path.exists(f):
+                    return None
+                h.update(open(f, "rb").read())
+            return float(kv["bytes"]) if h.hexdigest().startswith(kv.get("sha256", "?")) else None
+    return None
+
+
+def _stats(ts):
+    return dict(mean=sum(ts) / len(ts), median=statistics.median(ts), min=min(ts), n=len(ts))
 
 
 def _peaks():
@@ -80,14 +108,17 @@ class ClockSampler:
                     reasons=reasons, samples=len(rows), samples_in_timed_steps=len(timed), window=window)
 
 
-def _oracle_sample(cfg, rows, L=None):
-    """Times the oracle, as it stands, on `rows` token rows of the workload (whole path)."""
+def _oracle_sample(cfg, rows, L=None, parallel=False):
+    """Times the oracle, as it stands, on `rows` token rows of the workload (whole path).  parallel: the same source
+    built with -fopenmp, its loops over token rows on all the cores this process may use."""
     sys.path.insert(0, os.path.join(ROOT, "tests"))
     import oracle
     import parity
     from paper_2310_08041_b200 import synth
+    oracle.set_parallel(False)
     if L is None:
         L = parity.oracle_layer(cfg)
+    oracle.set_parallel(parallel)
     x = synth.activations(cfg, M=rows)
     t0 = time.perf_counter()
     q = oracle.reassemble_quant(x, L["gamma"], L["beta"], cfg.ln_eps, L["ptr"], L["src"], L["coef"], cfg.a_bits)
@@ -95,7 +126,29 @@ def _oracle_sample(cfg, rows, L=None):
     out = oracle.epilogue(acc, cfg.K, q["scale"], q["zero"], q["sum"], L["w_scale"], L["w_zero"], L["w_colsum"], None)
     oracle.cast_bf16(out)
     dt = time.perf_counter() - t0
+    oracle.set_parallel(False)
     return rows / dt, dt, L
+
+
+def _cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def _cpu_baseline(cfg, rows):
+    """The oracle on the host's cores: one thread on `rows` token rows, then all cores (OpenMP over token rows) on
+    as many rows per core.  The all-cores figure is the line's cpu_baseline value."""
+    cores = _cores()
+    v1, dt1, L = _oracle_sample(cfg, rows)
+    rows_all = rows * min(cores, 16)
+    os.environ["OMP_NUM_THREADS"] = str(cores)
+    vN, dtN, _ = _oracle_sample(cfg, rows_all, L, parallel=True)
+    return {"value": vN, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {rows_all} token rows of {cfg.name}, whole path, OpenMP over token rows, {dtN:.1f} s",
+            "single_thread": {"value": v1, "cores": 1,
+                              "sample": f"first {rows} token rows of {cfg.name}, whole path, {dt1:.1f} s"}}
 
 
 def run_reference(args):
@@ -175,7 +228,7 @@ def run_gpu(args):
     out = torch.empty((M, N), dtype=out_dtype, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
 
-    MID_EVERY = 4
+    MID_EVERY = 2
 
     def step(evs=None, mid=False):
         # the two calls of qllm_layer_forward.  Every MID_EVERY-th timed step records an event between them,
@@ -197,23 +250,42 @@ def run_gpu(args):
         step()
     barrier()
     assert B.qllm_poll_status() == 0, "device-side wait timed out during warm-up"
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    n0 = B.qllm_launch_count()
-    barrier()
+    # The timed region is K steps between a barrier + synchronize on both sides.  A region shorter than half a
+    # second would see no sample of the 100 ms clock sampler, so it is repeated (same K steps, same bracketing)
+    # until the rounds add up to that; every round's steps count.
+    t_pre, t_gemm, t_step, t_b2b = [], [], [], []
+    launches = 0
+    rounds = 0
     t_start = time.time()
-    for i in range(args.steps):
-        flush.zero_()                  # L2 flush between timed iterations (not inside the event pairs)
-        step(events[i], mid=(i % MID_EVERY == 0))
-    barrier()
+    while True:
+        events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        n0 = B.qllm_launch_count()
+        barrier()
+        for i in range(args.steps):
+            flush.zero_()                  # L2 flush between timed iterations (not inside the event pairs)
+            step(events[i], mid=(i % MID_EVERY == 0))
+        barrier()
+        if rounds == 0:
+            launches = B.qllm_launch_count() - n0
+        rounds += 1
+        for i, e in enumerate(events):
+            t = e[0].elapsed_time(e[2])
+            t_step.append(t)
+            if i % MID_EVERY == 0:
+                t_pre.append(e[0].elapsed_time(e[1]))
+                t_gemm.append(e[1].elapsed_time(e[2]))
+            else:
+                t_b2b.append(t)
+        more = time.time() - t_start < 0.6 and rounds < 5000
+        if world > 1:
+            flag = torch.tensor([1 if more else 0], device=dev)
+            dist.broadcast(flag, 0)
+            more = bool(flag.item())
+        if not more:
+            break
     t_end = time.time()
-    launches = B.qllm_launch_count() - n0
     assert B.qllm_poll_status() == 0, "device-side wait timed out"
-    halves = events[::MID_EVERY]
-    t_pre = [e[0].elapsed_time(e[1]) for e in halves]
-    t_gemm = [e[1].elapsed_time(e[2]) for e in halves]
-    t_step = [e[0].elapsed_time(e[2]) for e in events]
     ms_step = sum(t_step) / len(t_step)
-    t_b2b = [t for i, t in enumerate(t_step) if i % MID_EVERY != 0]
     ms_b2b = sum(t_b2b) / len(t_b2b) if t_b2b else ms_step
 
     # end to end through the host-buffer entry point: H2D of x and D2H of out inside the timed region
@@ -258,17 +330,20 @@ def run_gpu(args):
             roofline = {"kernel": "qllm_qgemm call: qgemm_decode_kernel (weight streaming)", "bound": "hbm",
                         "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                         "peak_source": f"{peaks['source']} STREAM-style copy", "ms": ms_gemm, "bytes": gemm_bytes,
-                        "traffic": NCU_TRAFFIC.get((cfg.name, M))}
+                        "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS,
+                        "traffic": _traffic("qgemm_decode_kernel", cfg.name, M)}
         else:
             expand = (cfg.a_bits == 4 or cfg.w_bits == 4) and M >= 385
             roofline = {"kernel": "qllm_layer_qgemm: " + ("join of the side-stream weight expansion + " if expand and cfg.w_bits == 4 else "") +
                                   "qgemm_tc2_kernel (tcgen05 kind::i8, cta_group::2, byte lanes) + dequant epilogue",
                         "bound": "tensor", "achieved": tops, "peak": int8_peak, "unit": "TOP/s", "frac": tops / int8_peak,
                         "peak_source": f"2 x {peaks['source']} bf16 burst ({peaks['bf16_burst']} TFLOP/s); nominal int8:bf16 = 2",
-                        "frac_of_nominal_4500": tops / 4500.0, "ms": ms_gemm, "traffic": NCU_TRAFFIC.get((cfg.name, M))}
+                        "frac_of_nominal_4500": tops / 4500.0, "ms": ms_gemm,
+                        "traffic": _traffic("qgemm_tc2_kernel", cfg.name, M)}
         line = {
             "metric": METRIC, "value": world * M / (ms_step_w * 1e-3), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step_w, "higher_is_better": True,
+            "steps": args.steps, "timed_rounds": rounds, "warmup": args.warmup, "ms_per_step": ms_step_w,
+            "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u8",
             "data": "synthetic",
             "config": {"workload": f"{cfg.name}: M={M} K={K} N={N} W{cfg.w_bits}A{cfg.a_bits} x=bf16 out=bf16 per GPU",
@@ -279,21 +354,58 @@ def run_gpu(args):
             "gpu_launches": int(launches),
             "clocks": clocks,
             "roofline": roofline,
-            "kernels": {"reassemble_quant": {"ms": ms_pre, "GB/s": pre_bytes / (ms_pre * 1e-3) / 1e9,
+            "ms_per_step_stats": _stats(t_step),
+            "ms_x_sm_mhz": (ms_step_w * clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
+            "kernels": {"reassemble_quant": {"ms": ms_pre, "ms_stats": _stats(t_pre),
+                                             "GB/s": pre_bytes / (ms_pre * 1e-3) / 1e9,
                                              "frac_hbm": pre_bytes / (ms_pre * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                             "frac_of_nominal_8000": pre_bytes / (ms_pre * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
                                              "bytes": pre_bytes},
-                        "qgemm": {"ms": ms_gemm, "TOP/s": tops},
-                        "timed_on": f"every {MID_EVERY}th timed step (event between the two calls)",
+                        "qgemm": {"ms": ms_gemm, "ms_stats": _stats(t_gemm), "TOP/s": tops},
+                        "timed_on": f"every {MID_EVERY}nd timed step (event between the two calls)",
                         "ms_per_step_without_that_event": ms_b2b},
         }
         if world == 1 and not args.no_cpu_baseline:
-            sys.path.insert(0, os.path.join(ROOT, "tests"))
-            rows = args.ref_rows or 512
-            v, dt, _ = _oracle_sample(cfg, rows)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": f"first {rows} token rows of {cfg.name}, whole path, {dt:.1f} s"}
+            line["cpu_baseline"] = _cpu_baseline(cfg, args.ref_rows or 384)
         print(json.dumps(line))
     layer.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def launch_ranks(n, argv):
+    """Starts n ranks of this script on this node (rank r on GPU r), as the multi-GPU contract does."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def run_stub(args):
+    """The rank plumbing of run_gpu without a GPU: gloo, a stand-in step whose time depends on the rank, the
+    max-over-ranks reduction and rank 0's line.  Tokens per rank are the sharding module's."""
+    import torch
+    import torch.distributed as dist
+    from paper_2310_08041_b200 import shard
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    M = 64
+    t = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        time.sleep(0.001 * (rank + 1))
+        if i >= args.warmup:
+            t.append((time.perf_counter() - t0) * 1e3)
+    ms = sum(t) / len(t)
+    ms_w = shard.max_over_ranks(ms) if world > 1 else ms
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": world * M / (ms_w * 1e-3), "unit": UNIT, "n_gpus": world,
+                          "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_w, "stub": True,
+                          "scaling": "weak", "config": {"parallelism": f"tokens x{world}"}}))
     if world > 1:
         dist.destroy_process_group()
 
@@ -307,9 +419,20 @@ def main():
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c2_w4a8"])
     ap.add_argument("--ref-rows", type=int, default=0, help="token rows of the oracle sample (0 = auto)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stub", action="store_true",
+                    help="no GPU: gloo ranks and a stand-in step, to exercise the launcher and the reduction")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is None and args.gpus > 1:
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))    # one process per GPU, this script again in each
+    if int(world_env or 1) != args.gpus:
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world_env}: refusing to print a line\n")
+        sys.exit(2)
+    if args.stub:
+        run_stub(args)
     else:
         run_gpu(args)
 

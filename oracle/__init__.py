@@ -20,22 +20,36 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "qllm_oracle.cpp")
 _LIB = os.path.join(_HERE, "libqllm_oracle.so")
+_LIB_OMP = os.path.join(_HERE, "libqllm_oracle_omp.so")
 _lib = None
+_parallel = False
 
 
-def build(force: bool = False) -> str:
-    """Compile the oracle with g++ (-O2, no threading, no fast-math)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        tmp = _LIB + ".tmp.%d" % os.getpid()
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-o", tmp, _SRC])
-        os.replace(tmp, _LIB)
-    return _LIB
+def build(force: bool = False, parallel: bool = False) -> str:
+    """Compile the oracle with g++ (-O2, no fast-math).  The default build is single-threaded: the OpenMP pragmas
+    on the loops over token rows are ignored.  parallel=True makes a second library with -fopenmp, in which
+    those loops (and nothing else) run on all cores; it exists for the benchmark's all-cores baseline."""
+    target = _LIB_OMP if parallel else _LIB
+    if force or not os.path.exists(target) or os.path.getmtime(target) < os.path.getmtime(_SRC):
+        tmp = target + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC"] + (["-fopenmp"] if parallel else []) +
+                              ["-o", tmp, _SRC])
+        os.replace(tmp, target)
+    return target
+
+
+def set_parallel(flag: bool) -> None:
+    """Switch the wrappers between the single-threaded library (default) and the OpenMP one."""
+    global _lib, _parallel
+    if flag != _parallel:
+        _parallel = flag
+        _lib = None
 
 
 def lib():
     global _lib
     if _lib is None:
-        _lib = ctypes.CDLL(build())
+        _lib = ctypes.CDLL(build(parallel=_parallel))
         _lib.orc_theta_percentile.restype = ctypes.c_float
         _lib.orc_theta_for_extra.restype = ctypes.c_float
         _lib.orc_extra_channels.restype = ctypes.c_int64

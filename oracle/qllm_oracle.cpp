@@ -83,6 +83,7 @@ extern "C" {
 // ---------------------------------------------------------------------------
 int orc_layernorm(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                   const float* beta, double eps, double* y) {
+#pragma omp parallel for schedule(static)
     for (int64_t m = 0; m < M; ++m) {
         double s = 0.0;
         for (int k = 0; k < C; ++k) s += load_x(x, x_dtype, m * C + k);
@@ -123,6 +124,7 @@ int orc_channel_absmax(const double* y, int64_t M, int C, float* absmax) {
 // ---------------------------------------------------------------------------
 int orc_map_apply(const double* y, int64_t M, int C_in, int C_out, const int32_t* ptr,
                   const int32_t* src, const float* coef, double* xr) {
+#pragma omp parallel for schedule(static)
     for (int64_t m = 0; m < M; ++m)
         for (int c = 0; c < C_out; ++c) {
             double s = 0.0;
@@ -147,6 +149,7 @@ int orc_map_apply(const double* y, int64_t M, int C_in, int C_out, const int32_t
 int orc_quant_rows(const double* v, int64_t R, int C, int bits, uint8_t* codes, float* scale,
                    float* zero, int32_t* codesum, double* pre, double* zpre) {
     const double qmax = static_cast<double>((1 << bits) - 1);
+#pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < R; ++r) {
         const double* row = v + r * C;
         double lo = row[0], hi = row[0];
@@ -217,15 +220,17 @@ int orc_weight_transform(const float* W, int N, int C_in, int C_out, const int32
 // 64-bit accumulation; returns -1 if any value would not fit an int32.
 // ---------------------------------------------------------------------------
 int orc_int_matmul(const uint8_t* qa, const uint8_t* qw, int64_t M, int N, int K, int32_t* acc) {
+    int overflow = 0;
+#pragma omp parallel for schedule(static)
     for (int64_t m = 0; m < M; ++m)
         for (int n = 0; n < N; ++n) {
             int64_t s = 0;
             for (int k = 0; k < K; ++k)
                 s += static_cast<int64_t>(qa[m * K + k]) * static_cast<int64_t>(qw[static_cast<int64_t>(n) * K + k]);
-            if (s > std::numeric_limits<int32_t>::max()) return -1;
-            acc[m * N + n] = static_cast<int32_t>(s);
+            if (s > std::numeric_limits<int32_t>::max()) overflow = 1;
+            else acc[m * N + n] = static_cast<int32_t>(s);
         }
-    return 0;
+    return overflow ? -1 : 0;
 }
 
 // Same sum for a list of (m, n) pairs only: lets full-size problems be checked
@@ -252,6 +257,7 @@ int orc_int_matmul_at(const uint8_t* qa, const uint8_t* qw, int K, const int64_t
 int orc_epilogue(const int32_t* acc, int64_t M, int N, int K, const float* a_scale,
                  const float* a_zero, const int32_t* a_rowsum, const float* w_scale,
                  const float* w_zero, const int32_t* w_colsum, const float* bias, double* out) {
+#pragma omp parallel for schedule(static)
     for (int64_t m = 0; m < M; ++m) {
         int64_t za = static_cast<int64_t>(a_zero[m]);
         for (int n = 0; n < N; ++n) {
@@ -272,6 +278,7 @@ int orc_cast_f32(const double* v, int64_t n, float* out) {
     return 0;
 }
 int orc_cast_bf16(const double* v, int64_t n, uint16_t* out) {
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n; ++i) out[i] = round_to_bf16(v[i]);
     return 0;
 }

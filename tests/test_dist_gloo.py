@@ -59,3 +59,26 @@ def test_two_gloo_ranks_shard_and_reduce():
         assert total == M
         s0, n0 = token_shard(M, 0, world)
         assert np.all(marks[:n0] == 1) and np.all(marks[n0:] == 2)   # every row owned exactly once
+
+
+def test_bench_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` with no rendezvous in the environment starts two ranks itself; rank 0 prints one line
+    whose n_gpus is the world size and whose time is the slowest rank's.  (--stub: gloo and a stand-in step.)"""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "3", "--warmup", "1", "--stub"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["config"]["parallelism"] == "tokens x2"
+    assert d["ms_per_step"] >= 1.9                 # rank 1 sleeps 2 ms per step: the max, not rank 0's 1 ms
+    # a world size that contradicts --gpus prints no line
+    env2 = dict(env, WORLD_SIZE="1", RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "4", "--steps", "1", "--warmup", "1", "--stub"],
+                       capture_output=True, text=True, timeout=120, env=env2)
+    assert r.returncode != 0 and not [l for l in r.stdout.splitlines() if l.startswith("{")]
