@@ -184,17 +184,28 @@ int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, i
 
 }  // namespace
 
-int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
-               const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
-               int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
-               cudaStream_t st, bool may_allocate, const uint8_t* w_ready) {
-    int rc = check_gemm_shape(M, N, K, a_bits, w_bits);
+// Every argument check of the GEMM entry points, before anything is launched.
+int gemm_check_args(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
+                    const float* w_scale, const float* w_zero, const int32_t* w_colsum, const void* out, int64_t M,
+                    int N, int K, int a_bits, int w_bits, int out_dtype) {
+    const int rc = check_gemm_shape(M, N, K, a_bits, w_bits);
     if (rc != QLLM_OK) return rc;
     if (!dtype_ok(out_dtype)) return QLLM_ERR_DTYPE;
     if (M == 0) return QLLM_OK;
     if (!codes || !a_scale || !a_zero || !w_codes || !w_scale || !w_zero || !w_colsum || !out)
         return QLLM_ERR_NULL;
     if (!aligned16(codes) || !aligned16(w_codes) || !aligned16(out)) return QLLM_ERR_ALIGN;
+    return QLLM_OK;
+}
+
+int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
+               const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
+               int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
+               cudaStream_t st, bool may_allocate, const uint8_t* w_ready) {
+    int rc = gemm_check_args(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, out, M, N, K, a_bits, w_bits,
+                             out_dtype);
+    if (rc != QLLM_OK) return rc;
+    if (M == 0) return QLLM_OK;
     if (!a_rowsum) {
         if (!may_allocate) return QLLM_ERR_NULL;
         int32_t* scratch = nullptr;

@@ -131,6 +131,9 @@ int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, 
                const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
                int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
                cudaStream_t st, bool may_allocate, const uint8_t* w_ready = nullptr);
+int gemm_check_args(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
+                    const float* w_scale, const float* w_zero, const int32_t* w_colsum, const void* out, int64_t M,
+                    int N, int K, int a_bits, int w_bits, int out_dtype);
 int launch_rowsum(const uint8_t* codes, int64_t M, int K, int bits, int32_t* rowsum, cudaStream_t st);
 int launch_qgemm_plain(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
                        int w_bits, const EpilogueArgs& ep, cudaStream_t st);

@@ -45,15 +45,16 @@ extern "C" int qllm_qgemm_noalloc(const uint8_t* codes, const float* a_scale, co
                                   const int32_t* w_colsum, const float* bias, void* out, int64_t M, int N,
                                   int K, int a_bits, int w_bits, int out_dtype, void* stream) {
     using namespace qllm;
-    if (!bits_ok(a_bits) || !bits_ok(w_bits)) return QLLM_ERR_BITS;
-    if (M < 0 || N <= 0 || K <= 0) return QLLM_ERR_SHAPE;
-    if ((a_bits == 4 || w_bits == 4) && (K & 1)) return QLLM_ERR_SHAPE;
-    if (M > QLLM_NOALLOC_MAX_M) return QLLM_ERR_UNSUPPORTED;   // more rows than the fixed scratch holds
+    if (bits_ok(a_bits) && bits_ok(w_bits) && M > QLLM_NOALLOC_MAX_M && N > 0 && K > 0)
+        return QLLM_ERR_UNSUPPORTED;                            // more rows than the fixed scratch holds
+    // all of qllm_qgemm's argument checks first: a call that returns an error has launched nothing and has not
+    // touched the array every call shares
+    int rc = gemm_check_args(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, out, M, N, K, a_bits, w_bits,
+                             out_dtype);
+    if (rc != QLLM_OK) return rc;
     if (M == 0) return QLLM_OK;
-    if (!codes) return QLLM_ERR_NULL;
-    if (!aligned16(codes)) return QLLM_ERR_ALIGN;
     int32_t* rowsum = nullptr;
-    int rc = scratch_address(&rowsum);
+    rc = scratch_address(&rowsum);
     if (rc != QLLM_OK) return rc;
     // every one of the M entries is overwritten, so nothing left by an earlier call is read
     rc = launch_rowsum(codes, M, K, a_bits, rowsum, static_cast<cudaStream_t>(stream));
