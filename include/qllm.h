@@ -320,6 +320,13 @@ int qllm_last_cuda_error(void);
  * QLLM_ERR_TIMEOUT if a bounded wait inside a kernel expired since the last poll.
  * Synchronizes the device. */
 int qllm_poll_status(void);
+/* Exercises the expiry path of the bounded device-side waits (every mbarrier wait of the tensor-core GEMM
+ * kernels gives up after ~2^32 cycles, raises the status word and lets its CTA wind down; the paper has no
+ * counterpart).  Launches one warp that waits, with the same routine under a limit of 2^20 cycles, for a barrier
+ * nobody arrives on: the wait runs out, the status word is set, the kernel returns.  Nothing faults, traps or
+ * spins without bound.  *gave_up (device int) becomes 1.  Afterwards qllm_poll_status() returns
+ * QLLM_ERR_TIMEOUT once and QLLM_OK again; other calls are unaffected.  Asynchronous on `stream`. */
+int qllm_debug_wait_expiry(int* gave_up, void* stream);
 /* Number of kernel launches issued by this library in this process (all threads). */
 int64_t qllm_launch_count(void);
 

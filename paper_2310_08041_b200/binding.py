@@ -31,7 +31,7 @@ EXPORTS = [
     "qllm_layer_create", "qllm_layer_destroy", "qllm_layer_forward", "qllm_layer_forward_host",
     "qllm_layer_reassemble_quant", "qllm_layer_qgemm",
     "qllm_layer_workspace",
-    "qllm_status_string", "qllm_last_cuda_error", "qllm_poll_status", "qllm_launch_count",
+    "qllm_status_string", "qllm_last_cuda_error", "qllm_poll_status", "qllm_launch_count", "qllm_debug_wait_expiry",
 ]
 
 if not os.path.exists(LIB_PATH):
@@ -75,6 +75,7 @@ _lib.qllm_layer_workspace.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_
 _lib.qllm_status_string.argtypes = [_i]
 _lib.qllm_status_string.restype = ctypes.c_char_p
 _lib.qllm_launch_count.restype = _i64
+_lib.qllm_debug_wait_expiry.argtypes = [_vp, _vp]
 
 
 class QllmError(RuntimeError):
@@ -159,6 +160,11 @@ def qllm_calib_absmax(x, ln_gamma, ln_beta, absmax, ln_eps=1e-5, stream=None):
 
 def qllm_poll_status():
     return _lib.qllm_poll_status()
+
+
+def qllm_debug_wait_expiry(gave_up, stream=None):
+    """Runs a bounded device-side wait into its (short) limit; gave_up: device int32 tensor, set to 1."""
+    _check(_lib.qllm_debug_wait_expiry(_dp(gave_up), _stream(stream)))
 
 
 def qllm_launch_count():

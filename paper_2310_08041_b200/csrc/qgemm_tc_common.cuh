@@ -25,14 +25,17 @@ struct Abort {
     int* status;            // global status word of the library
 };
 
-__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, const Abort& ab) {
+// Waits for a phase of an mbarrier for at most `limit` cycles.  On expiry the CTA's abort flag and the library's
+// status word are set and the caller leaves its loop (false); a role that sees the flag set by another gives up too.
+__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, const Abort& ab,
+                                             long long limit = kWaitCycles) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t i = 1;; ++i) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 0) {
             if (*ab.flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > limit) {
                 *ab.flag = 1;
                 atomicExch(ab.status, QLLM_ERR_TIMEOUT);
                 return false;

@@ -142,3 +142,26 @@ def test_empty_and_status():
         B.qllm_qgemm(zb, z, z, zb, z, z, zi, None, z, 2, 8, 15, 4, 4)
     assert e.value.status == B.QLLM_ERR_SHAPE
     assert B.qllm_poll_status() == 0
+
+
+def test_bounded_wait_expiry_is_reported_once_and_harmless():
+    """A device-side wait that runs out raises the status word and returns; the host reads QLLM_ERR_TIMEOUT once,
+    then QLLM_OK, and the next GEMM is bit-exact.  The expiry is produced by a one-warp kernel that waits, under a
+    short limit, for a barrier nothing arrives on (the GEMM kernels themselves are not altered for the test)."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    assert B.qllm_poll_status() == 0
+    gave_up = torch.zeros(1, dtype=torch.int32, device=G.DEV)
+    B.qllm_debug_wait_expiry(gave_up)
+    torch.cuda.synchronize()                       # the launch returns
+    assert int(gave_up.item()) == 1
+    assert B.qllm_poll_status() == B.QLLM_ERR_TIMEOUT
+    assert B.qllm_poll_status() == 0               # reported once
+    M, N, K = 300, 384, 512
+    qa, qw = synth.random_codes(3, M, K, 8), synth.random_codes(4, N, K, 8)
+    acc = torch.zeros((M, N), dtype=torch.int32, device=G.DEV)
+    B.qllm_qgemm_acc(G.dev(qa), G.dev(qw), acc, M, N, K, 8, 8)
+    torch.cuda.synchronize()
+    assert np.array_equal(acc.cpu().numpy(), oracle.int_matmul(qa, qw))
+    assert B.qllm_poll_status() == 0
