@@ -201,17 +201,32 @@ int qllm_build_reassembly(const float* calib_absmax, int C, float theta,
                           int w_bits, qllm_reassembly_t** out);
 void qllm_free_reassembly(qllm_reassembly_t* h);
 
-/* The same builder with the distance of Eq. 5 in the bipartite matching: dist is a HOST float[C][C] table,
- * dist[i][j] = 1/4 ||y_i - y_j||^2 ||W_i - W_j||^2 over the calibration tokens (qllm_channel_distance computes it
- * on the device).  Nearest counterpart, tie rules and edge selection are those of qllm_build_reassembly with
- * dist[a][b] in place of |m_a - m_b|.  Eq. 5 is defined between undivided channels, so only one matching round
- * is possible: a threshold that needs a second round returns QLLM_ERR_UNSUPPORTED. */
-int qllm_build_reassembly_eq5(const float* calib_absmax, int C, float theta, const float* dist,
+/* The same builder with the distance of Eq. 5 in the bipartite matching (Sec. 4.1.2; the paper names these
+ * pairwise distances as the main cost of reassembly): D(i, j) = 1/4 ||y_i - y_j||^2 ||W_i - W_j||^2, y_i the
+ * column of channel i over the T calibration rows of the layer's input, W_i the weights of input channel i.
+ *  calib_y   DEVICE float[T][C]: the layer's input of the calibration tokens (qllm_layernorm_rows makes it)
+ *  W         host float[N][C] as above (copied to the device for the duration of the call)
+ *  stream    the device work (nearest-neighbour search: for every entry of set A the nearest entry of set B,
+ *            Appendix A step 2) runs there; the call waits for it.  Only those |A| edges come back to the host.
+ * Nearest counterpart, tie rules and edge selection are those of qllm_build_reassembly with D(a, b) in place of
+ * |m_a - m_b|; D is evaluated in float32.  Eq. 5 is defined between undivided channels, so only one matching
+ * round is possible: a threshold that needs a second round returns QLLM_ERR_UNSUPPORTED.  A row of distances
+ * without a finite value returns QLLM_ERR_MAP.  Offline step: allocates and frees device memory. */
+int qllm_build_reassembly_eq5(const float* calib_absmax, int C, float theta,
+                              const float* calib_y, int64_t T,
                               const float* W, int N,
                               const float* lr_A, const float* lr_B, int r,
-                              int w_bits, qllm_reassembly_t** out);
+                              int w_bits, void* stream, qllm_reassembly_t** out);
 
-/* Build-time device helpers for that table (asynchronous on stream; all pointers DEVICE).
+/* The builder driven by a caller-made distance table: dist is a HOST float[C][C], dist[a][b] takes the place of
+ * |m_a - m_b| (same rules, one round only, QLLM_ERR_MAP for a row without a finite value).  qllm_channel_distance
+ * makes the Eq. 5 table on the device when the whole table is wanted. */
+int qllm_build_reassembly_dist(const float* calib_absmax, int C, float theta, const float* dist,
+                               const float* W, int N,
+                               const float* lr_A, const float* lr_B, int r,
+                               int w_bits, qllm_reassembly_t** out);
+
+/* Build-time device helpers (asynchronous on stream; all pointers DEVICE).
  * qllm_layernorm_rows: y[t][c] = LayerNorm(x[t])[c] as float32, the linear layer's input of the calibration
  * tokens (x [T][C] in x_dtype, ln_beta may be NULL).
  * qllm_channel_distance: D[i][j] of Eq. 5 from y [T][C] and the layer's weights W [N][C] (output channel major,

@@ -223,12 +223,12 @@ class NeedsMoreRounds(Exception):
 
 
 def channel_distance(y, W):
-    """Eq. 5 table D[i][j] = 1/4 ||y_i - y_j||^2 ||W_i - W_j||^2 (float32, defined order).  y [T][C], W [N][C]."""
-    y = _c(y, np.float32); W = _c(W, np.float32)
+    """Eq. 5 table D[i][j] = 1/4 ||y_i - y_j||^2 ||W_i - W_j||^2 in fp64.  y [T][C] (fp64), W [N][C] (fp32)."""
+    y = _c(y, np.float64); W = _c(W, np.float32)
     T, C = y.shape
     N = W.shape[0]
     assert W.shape[1] == C
-    D = np.empty((C, C), np.float32)
+    D = np.empty((C, C), np.float64)
     lib().orc_channel_distance(_p(y), ctypes.c_int64(T), _p(W), ctypes.c_int(N), ctypes.c_int(C), _p(D))
     return D
 
@@ -245,7 +245,7 @@ def build_map(absmax, theta, dist=None):
         rc = lib().orc_build_map(_p(a), ctypes.c_int(C), ctypes.c_float(theta), _p(ptr), _p(src), _p(coef),
                                  ctypes.c_int64(cap), _p(stats))
     else:
-        d = _c(dist, np.float32)
+        d = _c(dist, np.float64)
         assert d.shape == (C, C)
         rc = lib().orc_build_map_dist(_p(a), ctypes.c_int(C), ctypes.c_float(theta), _p(d), _p(ptr), _p(src), _p(coef),
                                       ctypes.c_int64(cap), _p(stats))

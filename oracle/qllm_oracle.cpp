@@ -362,7 +362,7 @@ float orc_theta_for_extra(const float* absmax, int C, int extra) {
 // distance between two entries is |m_a - m_b|.  With it the distance between two undivided channels is
 // dist[a][b]; a second matching round would need distances between merged sets, which Eq. 5 does not define:
 // -4 is returned instead.
-static int build_map_impl(const float* absmax, int C, float theta, const float* dist, int32_t* ptr, int32_t* src,
+static int build_map_impl(const float* absmax, int C, float theta, const double* dist, int32_t* ptr, int32_t* src,
                           float* coef, int64_t nnz_cap, int64_t* stats) {
     if (!(theta > 0.f)) return -3;
     std::vector<Entry> list;
@@ -396,7 +396,7 @@ static int build_map_impl(const float* absmax, int C, float theta, const float* 
             double best = std::numeric_limits<double>::infinity();
             int bb = -1;
             for (int b : B) {
-                double d = dist ? static_cast<double>(dist[static_cast<int64_t>(list[a].members[0]) * C + list[b].members[0]])
+                double d = dist ? dist[static_cast<int64_t>(list[a].members[0]) * C + list[b].members[0]]
                                 : std::fabs(list[a].m - list[b].m);
                 if (d < best) { best = d; bb = b; }   // B ascending: first minimum = lowest position
             }
@@ -450,7 +450,7 @@ int orc_build_map(const float* absmax, int C, float theta, int32_t* ptr, int32_t
 }
 
 // The same builder with the distance of Eq. 5 between undivided channels, given as a C x C table.
-int orc_build_map_dist(const float* absmax, int C, float theta, const float* dist, int32_t* ptr, int32_t* src,
+int orc_build_map_dist(const float* absmax, int C, float theta, const double* dist, int32_t* ptr, int32_t* src,
                        float* coef, int64_t nnz_cap, int64_t* stats) {
     if (!dist) return -3;
     return build_map_impl(absmax, C, theta, dist, ptr, src, coef, nnz_cap, stats);
@@ -460,24 +460,23 @@ int orc_build_map_dist(const float* absmax, int C, float theta, const float* dis
 // Eq. 5: the output error of merging channels i and j,
 //     D(i, j) = || (x_i (W_i - W_j) + x_j (W_j - W_i)) / 2 ||_F^2 = 1/4 ||x_i - x_j||^2 ||W_i - W_j||^2,
 // x_i the column of channel i over the T calibration rows of y (the linear layer's input), W_i the
-// weights of input channel i over the N outputs.  The table decides an argmin (the nearest channel), so it
-// is computed in the precision and order the product uses: float32, rows taken in order with one fused
-// multiply-add each,   dx = fma(e, e, dx), e = y[t][i] - y[t][j];   D = (0.25f * dx) * dw.
+// weights of input channel i over the N outputs.  Plain definition in fp64.
 // y: [T][C], w: [N][C] (output channel major), D: [C][C].
 // ---------------------------------------------------------------------------
-void orc_channel_distance(const float* y, int64_t T, const float* w, int N, int C, float* D) {
+void orc_channel_distance(const double* y, int64_t T, const float* w, int N, int C, double* D) {
     for (int i = 0; i < C; ++i) {
         for (int j = 0; j < C; ++j) {
-            float dx = 0.f, dw = 0.f;
+            double dx = 0.0, dw = 0.0;
             for (int64_t t = 0; t < T; ++t) {
-                const float e = y[t * C + i] - y[t * C + j];
-                dx = std::fmaf(e, e, dx);
+                const double e = y[t * C + i] - y[t * C + j];
+                dx += e * e;
             }
             for (int n = 0; n < N; ++n) {
-                const float e = w[static_cast<int64_t>(n) * C + i] - w[static_cast<int64_t>(n) * C + j];
-                dw = std::fmaf(e, e, dw);
+                const double e = static_cast<double>(w[static_cast<int64_t>(n) * C + i]) -
+                                 static_cast<double>(w[static_cast<int64_t>(n) * C + j]);
+                dw += e * e;
             }
-            D[static_cast<int64_t>(i) * C + j] = (0.25f * dx) * dw;
+            D[static_cast<int64_t>(i) * C + j] = 0.25 * dx * dw;
         }
     }
 }

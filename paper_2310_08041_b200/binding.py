@@ -25,7 +25,7 @@ QLLM_F32, QLLM_BF16 = 0, 1
 # every symbol include/qllm.h declares
 EXPORTS = [
     "qllm_reassemble_quant", "qllm_qgemm", "qllm_qgemm_noalloc", "qllm_qgemm_acc", "qllm_calib_absmax",
-    "qllm_build_reassembly", "qllm_build_reassembly_eq5", "qllm_layernorm_rows", "qllm_channel_distance", "qllm_free_reassembly", "qllm_reassembly_map",
+    "qllm_build_reassembly", "qllm_build_reassembly_eq5", "qllm_build_reassembly_dist", "qllm_layernorm_rows", "qllm_channel_distance", "qllm_free_reassembly", "qllm_reassembly_map",
     "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map", "qllm_fold_previous",
     "qllm_theta_percentile", "qllm_theta_for_extra", "qllm_search_theta",
     "qllm_layer_create", "qllm_layer_destroy", "qllm_layer_forward", "qllm_layer_forward_host",
@@ -47,7 +47,8 @@ _lib.qllm_qgemm_noalloc.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp,
 _lib.qllm_qgemm_acc.argtypes = [_vp, _vp, _vp, _i64, _i, _i, _i, _i, _vp]
 _lib.qllm_calib_absmax.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp]
 _lib.qllm_build_reassembly.argtypes = [_vp, _i, _f, _vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(_vp)]
-_lib.qllm_build_reassembly_eq5.argtypes = [_vp, _i, _f, _vp, _vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(_vp)]
+_lib.qllm_build_reassembly_dist.argtypes = [_vp, _i, _f, _vp, _vp, _i, _vp, _vp, _i, _i, ctypes.POINTER(_vp)]
+_lib.qllm_build_reassembly_eq5.argtypes = [_vp, _i, _f, _vp, _i64, _vp, _i, _vp, _vp, _i, _i, _vp, ctypes.POINTER(_vp)]
 _lib.qllm_layernorm_rows.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp]
 _lib.qllm_channel_distance.argtypes = [_vp, _i64, _vp, _i, _i, _vp, _vp]
 _lib.qllm_free_reassembly.argtypes = [_vp]
@@ -286,8 +287,10 @@ def qllm_channel_distance(y, W, D, stream=None):
     _check(_lib.qllm_channel_distance(_dp(y), T, _dp(W), W.shape[0], C, _dp(D), _stream(stream)))
 
 
-def qllm_build_reassembly(calib_absmax, theta, W, lr_A=None, lr_B=None, w_bits=4, dist=None):
-    """dist: optional host float32 [C][C] table of Eq. 5 distances (then qllm_build_reassembly_eq5 is called)."""
+def qllm_build_reassembly(calib_absmax, theta, W, lr_A=None, lr_B=None, w_bits=4, dist=None, calib_y=None, stream=None):
+    """dist: optional host float32 [C][C] distance table (qllm_build_reassembly_dist).  calib_y: optional DEVICE
+    float32 tensor [T][C], the layer's input of the calibration tokens: the matching then uses the Eq. 5 distance,
+    evaluated on the device (qllm_build_reassembly_eq5)."""
     a = np.ascontiguousarray(calib_absmax, np.float32)
     W = np.ascontiguousarray(W, np.float32)
     N, C = W.shape
@@ -299,13 +302,17 @@ def qllm_build_reassembly(calib_absmax, theta, W, lr_A=None, lr_B=None, w_bits=4
         r = lr_A.shape[1]
         assert lr_A.shape == (C, r) and lr_B.shape == (r, N)
     h = _vp()
-    if dist is None:
+    if calib_y is not None:
+        assert dist is None and tuple(calib_y.shape[1:]) == (C,)
+        _check(_lib.qllm_build_reassembly_eq5(_hp(a), C, theta, _dp(calib_y), calib_y.shape[0], _hp(W), N, _hp(lr_A),
+                                              _hp(lr_B), r, w_bits, _stream(stream), ctypes.byref(h)))
+    elif dist is None:
         _check(_lib.qllm_build_reassembly(_hp(a), C, theta, _hp(W), N, _hp(lr_A), _hp(lr_B), r, w_bits, ctypes.byref(h)))
     else:
         d = np.ascontiguousarray(dist, np.float32)
         assert d.shape == (C, C)
-        _check(_lib.qllm_build_reassembly_eq5(_hp(a), C, theta, _hp(d), _hp(W), N, _hp(lr_A), _hp(lr_B), r, w_bits,
-                                              ctypes.byref(h)))
+        _check(_lib.qllm_build_reassembly_dist(_hp(a), C, theta, _hp(d), _hp(W), N, _hp(lr_A), _hp(lr_B), r, w_bits,
+                                               ctypes.byref(h)))
     return Reassembly(h, C, N)
 
 

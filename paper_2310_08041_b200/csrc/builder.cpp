@@ -15,7 +15,15 @@
 #include <thread>
 #include <vector>
 
+#include <cuda_runtime.h>
+
 #include "../../include/qllm.h"
+
+namespace qllm {
+// channel_distance.cu: nearest channel of B for every channel of A under Eq. 5, on the device
+int eq5_nearest_device(const float* y, int64_t T, const float* w, int N, int C, const int* a_idx, int nA,
+                       const int* b_idx, int nB, int* best, float* best_d, cudaStream_t st);
+}
 
 struct qllm_reassembly {
     int C = 0, N = 0, w_bits = 0;
@@ -44,6 +52,15 @@ struct Slot {
     double m;      // calibration maximum (mean over members for a merged set)
 };
 
+// Calibration data on the device for the Eq. 5 distance: y [T][C] (the layer's input), w [N][C].
+struct Eq5Device {
+    const float* y;
+    int64_t T;
+    const float* w;
+    int N;
+    cudaStream_t st;
+};
+
 struct BKey {
     double m;
     int pos;
@@ -52,10 +69,12 @@ struct BKey {
 
 // One round of bipartite soft matching on `slots`; merges up to `need` A-slots into
 // their nearest B-slot.  Returns the number of merges done (0 = no eligible pair).
-// dist (optional): C x C table of Eq. 5 distances between undivided channels; the nearest b of an a is then
-// found by a scan over B on that table (the table has no order to search in).
+// dist (optional): C x C table of distances between undivided channels; the nearest b of an a is then found by a
+// scan over B on that table (the table has no order to search in).  dev (optional): the Eq. 5 distance is
+// evaluated on the device from calibration data and only the |A| nearest-neighbour edges come back.
+// A negative return is a status code.
 int64_t matching_round(std::vector<Slot>& slots, std::vector<int>& next_member,
-                       const float* absmax, int64_t need, const float* dist, int C) {
+                       const float* absmax, int64_t need, const float* dist, const Eq5Device* dev, int C) {
     const int L = int(slots.size());
     std::vector<int> A;
     std::vector<BKey> B;
@@ -69,7 +88,21 @@ int64_t matching_round(std::vector<Slot>& slots, std::vector<int>& next_member,
 
     struct Edge { double d; int a; int b; };
     std::vector<Edge> edges(A.size());
-    if (dist) {
+    if (dev) {
+        std::vector<int> Bpos, a_idx, b_idx;              // B in list order: ties go to the lowest position
+        for (int p = 1; p < L; p += 2)
+            if (!slots[p].sub) { Bpos.push_back(p); b_idx.push_back(slots[p].head); }
+        for (int a : A) a_idx.push_back(slots[a].head);
+        std::vector<int> best(A.size(), -1);
+        std::vector<float> best_d(A.size(), 0.f);
+        const int rc = qllm::eq5_nearest_device(dev->y, dev->T, dev->w, dev->N, C, a_idx.data(), int(a_idx.size()),
+                                                b_idx.data(), int(b_idx.size()), best.data(), best_d.data(), dev->st);
+        if (rc != QLLM_OK) return rc;
+        for (size_t i = 0; i < A.size(); ++i) {
+            if (best[i] < 0 || !std::isfinite(best_d[i])) return QLLM_ERR_MAP;   // no usable distance in the row
+            edges[i] = {double(best_d[i]), A[i], Bpos[size_t(best[i])]};
+        }
+    } else if (dist) {
         std::vector<int> Bpos;                            // B in list order: ties go to the lowest position
         for (int p = 1; p < L; p += 2)
             if (!slots[p].sub) Bpos.push_back(p);
@@ -81,10 +114,11 @@ int64_t matching_round(std::vector<Slot>& slots, std::vector<int>& next_member,
                 const double d = double(row[slots[p].head]);
                 if (d < best) { best = d; best_pos = p; }
             }
+            if (best_pos < 0) return QLLM_ERR_MAP;        // every distance of the row is NaN or +inf
             edges[i] = {best, A[i], best_pos};
         }
     }
-    for (size_t i = 0; i < A.size() && !dist; ++i) {
+    for (size_t i = 0; i < A.size() && !dist && !dev; ++i) {
         const int a = A[i];
         const double ma = slots[a].m;
         // first key with m >= ma
@@ -131,7 +165,7 @@ int64_t matching_round(std::vector<Slot>& slots, std::vector<int>& next_member,
     return keep;
 }
 
-int build_map(const float* absmax, int C, float theta, const float* dist, qllm_reassembly& h) {
+int build_map(const float* absmax, int C, float theta, const float* dist, const Eq5Device* dev, qllm_reassembly& h) {
     std::vector<Slot> slots;
     slots.reserve(size_t(C) + 64);
     int64_t E = 0;
@@ -144,8 +178,9 @@ int build_map(const float* absmax, int C, float theta, const float* dist, qllm_r
     std::vector<int> next_member(size_t(C), -1);
     int64_t need = E, rounds = 0;
     while (need > 0) {
-        if (dist && rounds > 0) return QLLM_ERR_UNSUPPORTED;   // Eq. 5 is defined between undivided channels only
-        int64_t done = matching_round(slots, next_member, absmax, need, dist, C);
+        if ((dist || dev) && rounds > 0) return QLLM_ERR_UNSUPPORTED;   // Eq. 5 is defined between undivided channels only
+        int64_t done = matching_round(slots, next_member, absmax, need, dist, dev, C);
+        if (done < 0) return int(done);
         if (done == 0) return QLLM_ERR_INFEASIBLE;
         need -= done;
         ++rounds;
@@ -242,7 +277,8 @@ void transform_and_quantize(const float* W, int N, int C, const float* lrA, cons
 
 extern "C" {
 
-static int build_reassembly_impl(const float* calib_absmax, int C, float theta, const float* dist, const float* W,
+static int build_reassembly_impl(const float* calib_absmax, int C, float theta, const float* dist,
+                                 const Eq5Device* dev, const float* W,
                                  int N, const float* lr_A, const float* lr_B, int r, int w_bits,
                                  qllm_reassembly_t** out) {
     if (!calib_absmax || !W || !out) return QLLM_ERR_NULL;
@@ -258,7 +294,7 @@ static int build_reassembly_impl(const float* calib_absmax, int C, float theta, 
     h->C = C; h->N = N; h->w_bits = w_bits;
     int rc;
     try {
-        rc = build_map(calib_absmax, C, theta, dist, *h);
+        rc = build_map(calib_absmax, C, theta, dist, dev, *h);
         if (rc == QLLM_OK) transform_and_quantize(W, N, C, lr_A, lr_B, r, w_bits, *h);
     } catch (const std::bad_alloc&) {
         rc = QLLM_ERR_NOMEM;
@@ -271,14 +307,35 @@ static int build_reassembly_impl(const float* calib_absmax, int C, float theta, 
 int qllm_build_reassembly(const float* calib_absmax, int C, float theta, const float* W, int N,
                           const float* lr_A, const float* lr_B, int r, int w_bits,
                           qllm_reassembly_t** out) {
-    return build_reassembly_impl(calib_absmax, C, theta, nullptr, W, N, lr_A, lr_B, r, w_bits, out);
+    return build_reassembly_impl(calib_absmax, C, theta, nullptr, nullptr, W, N, lr_A, lr_B, r, w_bits, out);
 }
 
-int qllm_build_reassembly_eq5(const float* calib_absmax, int C, float theta, const float* dist, const float* W,
-                              int N, const float* lr_A, const float* lr_B, int r, int w_bits,
-                              qllm_reassembly_t** out) {
+int qllm_build_reassembly_dist(const float* calib_absmax, int C, float theta, const float* dist, const float* W,
+                               int N, const float* lr_A, const float* lr_B, int r, int w_bits,
+                               qllm_reassembly_t** out) {
     if (!dist) return QLLM_ERR_NULL;
-    return build_reassembly_impl(calib_absmax, C, theta, dist, W, N, lr_A, lr_B, r, w_bits, out);
+    return build_reassembly_impl(calib_absmax, C, theta, dist, nullptr, W, N, lr_A, lr_B, r, w_bits, out);
+}
+
+int qllm_build_reassembly_eq5(const float* calib_absmax, int C, float theta, const float* calib_y, int64_t T,
+                              const float* W, int N, const float* lr_A, const float* lr_B, int r, int w_bits,
+                              void* stream, qllm_reassembly_t** out) {
+    if (!calib_y || !W) return QLLM_ERR_NULL;
+    if (T <= 0 || C <= 0 || N <= 0) return QLLM_ERR_SHAPE;
+    // the weights beside the calibration rows on the device, for the duration of the build
+    float* w_dev = nullptr;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMalloc(&w_dev, sizeof(float) * size_t(N) * size_t(C)) != cudaSuccess) { cudaGetLastError(); return QLLM_ERR_NOMEM; }
+    if (cudaMemcpyAsync(w_dev, W, sizeof(float) * size_t(N) * size_t(C), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(w_dev);
+        return QLLM_ERR_CUDA;
+    }
+    const Eq5Device dev{calib_y, T, w_dev, N, st};
+    const int rc = build_reassembly_impl(calib_absmax, C, theta, nullptr, &dev, W, N, lr_A, lr_B, r, w_bits, out);
+    cudaStreamSynchronize(st);
+    cudaFree(w_dev);
+    return rc;
 }
 
 void qllm_free_reassembly(qllm_reassembly_t* h) { delete h; }

@@ -123,6 +123,9 @@ int launch_reassemble_quant_generic(const void* x, int x_dtype, int64_t M, int C
 // y[t][c] = LayerNorm(x[t])[c] in fp32 (build-time helper)
 int launch_layernorm_rows(const void* x, int x_dtype, int64_t T, int C, const float* gamma, const float* beta,
                           float eps, float* y, cudaStream_t st);
+// Eq. 5 nearest-B search on the device for the host builder (see channel_distance.cu)
+int eq5_nearest_device(const float* y, int64_t T, const float* w, int N, int C, const int* a_idx, int nA,
+                       const int* b_idx, int nB, int* best, float* best_d, cudaStream_t st);
 int launch_calib_absmax(const void* x, int x_dtype, int64_t M, int C, const float* gamma,
                         const float* beta, float eps, float* absmax, cudaStream_t st);
 int launch_expand_codes(const uint8_t* packed, int64_t rows, int K, uint8_t* bytes, cudaStream_t st);

@@ -107,14 +107,14 @@ def test_theta_helpers_match():
 
 
 def test_builder_with_eq5_table_matches_oracle():
-    """Host builder driven by an Eq. 5 distance table (here the oracle's table: the device kernel that makes it
-    is checked bit for bit in the GPU tests) against the oracle's table-driven builder."""
+    """Host builder driven by a distance table (here the oracle's Eq. 5 table, rounded to the float32 the builder
+    takes) against the oracle's table-driven builder."""
     cfg = synth.CONFIGS["c2"].scaled(M=32, K=256, N=48, n_outlier=4, calib_tokens=24)
     g, b = synth.layernorm_params(cfg)
-    y = oracle.layernorm(synth.calibration_tokens(cfg), g, b, cfg.ln_eps).astype(np.float32)
+    y = oracle.layernorm(synth.calibration_tokens(cfg), g, b, cfg.ln_eps)
     absmax = oracle.channel_absmax(y)
     W = synth.weights(cfg)
-    D = oracle.channel_distance(y, W)
+    D = oracle.channel_distance(y, W).astype(np.float32)   # the table the product's builder takes is float32: both sides get these values
     theta = oracle.theta_percentile(absmax, 0.97)
     ptr, src, coef, st = oracle.build_map(absmax, theta, dist=D)
     assert st["E"] > 0 and st["rounds"] == 1
@@ -133,3 +133,9 @@ def test_builder_with_eq5_table_matches_oracle():
         oracle.build_map(big, theta, dist=D)
     with pytest.raises(B.QllmError):
         B.qllm_build_reassembly(big, theta, W, w_bits=4, dist=D)
+    # a row of the table without a finite distance is refused, not indexed with
+    bad = D.copy()
+    bad[:, :] = np.inf
+    with pytest.raises(B.QllmError) as e:
+        B.qllm_build_reassembly(absmax, theta, W, w_bits=4, dist=bad)
+    assert e.value.status == B.QLLM_ERR_MAP

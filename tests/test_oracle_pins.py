@@ -480,7 +480,7 @@ def test_channel_distance_is_eq5_and_equals_the_error_of_the_merge():
     y64, W64 = y.astype(np.float64), W.astype(np.float64)
     ref = np.array([[0.25 * ((y64[:, i] - y64[:, j]) ** 2).sum() * ((W64[:, i] - W64[:, j]) ** 2).sum()
                      for j in range(C)] for i in range(C)])
-    np.testing.assert_allclose(D, ref, rtol=2e-5, atol=0)
+    np.testing.assert_allclose(D, ref, rtol=1e-12, atol=0)
     assert np.array_equal(D, D.T) and np.all(np.diag(D) == 0)
     # Eq. 5 is the output error of assembling the two channels (Eq. 4): build that map by hand and measure it
     i, j = 3, 10
