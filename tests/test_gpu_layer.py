@@ -43,9 +43,21 @@ def test_layer_forward_matches_oracle(name, kw, out_dtype):
     layer.forward(G.dev_x(x), out)
     torch.cuda.synchronize()
     assert B.qllm_poll_status() == 0
-    # activations: the flip rule
+    # activations: the flip rule, on the direct entry point and on what the layer's own pass left in its workspace
+    # (larger batches may hold one code per byte there)
     ref_q = oracle.reassemble_quant(x, L["gamma"], L["beta"], cfg.ln_eps, L["ptr"], L["src"], L["coef"], cfg.a_bits, want_pre=True)
-    got = G.run_reassemble_quant(x, L["gamma"], L["beta"], cfg.ln_eps, L["ptr"], L["src"], L["coef"], cfg.a_bits)
+    direct = G.run_reassemble_quant(x, L["gamma"], L["beta"], cfg.ln_eps, L["ptr"], L["src"], L["coef"], cfg.a_bits)
+    parity.check_activation_codes(direct["codes"], direct["scale"], direct["zero"], direct["rowsum"], ref_q, cfg.a_bits)
+    pc, ps, pz, pr, lanes = layer.workspace_ptrs()
+
+    def from_dev(p, shape, typestr):
+        class View:
+            __cuda_array_interface__ = dict(shape=tuple(shape), typestr=typestr, data=(int(p), False), version=2)
+        return torch.as_tensor(View(), device=G.DEV).cpu().numpy().copy()
+
+    wcodes = from_dev(pc, (cfg.M, cfg.K if lanes == 8 else cfg.K // 2), "|u1")
+    got = dict(codes=parity.unpack_codes(wcodes, 4) if lanes == 4 else wcodes, scale=from_dev(ps, (cfg.M,), "<f4"),
+               zero=from_dev(pz, (cfg.M,), "<f4"), rowsum=from_dev(pr, (cfg.M,), "<i4"))
     parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref_q, cfg.a_bits)
     # outputs: the oracle's GEMM + epilogue on the codes the GPU produced (identical codes)
     acc = oracle.int_matmul(got["codes"], L["w_codes"])
@@ -122,10 +134,13 @@ def test_layer_full_size_two_halves_sampled(name):
                                     L["w_scale"][n:n + 1], L["w_zero"][n:n + 1], L["w_colsum"][n:n + 1])[0, 0]
                     for a, m, n in zip(acc, ms, ns)])
     parity.check_output(G.bf16_bits(out.cpu())[ms, ns], ref, "bf16")
-    # the host-buffer entry point (chunked and overlapped at this size) returns the same bytes
+    # the host-buffer entry point (chunked and overlapped at this size) returns the same bytes as the one call with
+    # device buffers
     xh = torch.from_numpy(x.view(np.int16)).pin_memory()
     oh = torch.zeros((M, N), dtype=torch.bfloat16).pin_memory()
     layer.forward_host(xh, oh, M)
+    layer.forward(xd, out)
+    torch.cuda.synchronize()
     diff = oh.view(torch.int16) != out.cpu().view(torch.int16)
     assert not bool(diff.any()), (f"{int(diff.sum())} entries differ, rows {torch.nonzero(diff.any(1)).flatten()[:8].tolist()}"
                                   f" cols {torch.nonzero(diff.any(0)).flatten()[:8].tolist()}")
@@ -233,4 +248,56 @@ def test_decode_calls_back_to_back_see_their_own_tokens():
     assert B.qllm_poll_status() == 0
     for i, o in enumerate(outs):
         assert torch.equal(o, refs[i % 3]), i
+    layer.destroy()
+
+
+@pytest.mark.parametrize("name,kw", [("c2", dict(M=600, N=272)), ("c4", dict(M=150, N=144))])
+def test_product_pipeline_end_to_end_as_the_benchmark_runs_it(name, kw):
+    """Calibration statistic on the GPU -> threshold -> host builder -> layer -> forward, nothing taken from the
+    oracle on the way (the benchmark's set-up).  The oracle then runs on the SAME statistic: same threshold, same
+    map, same weight codes; activation codes under the flip rule; outputs from the oracle's integer product and
+    epilogue on the codes the GPU produced."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    cfg = synth.CONFIGS[name].scaled(**kw)
+    gamma, beta = synth.layernorm_params(cfg)
+    absmax = torch.zeros(cfg.K, dtype=torch.float32, device=G.DEV)
+    B.qllm_calib_absmax(G.dev_x(synth.calibration_tokens(cfg)), G.dev(gamma), None, absmax, ln_eps=cfg.ln_eps)
+    am = absmax.cpu().numpy()
+    theta = B.qllm_theta_percentile(am, 0.99)
+    W = synth.weights(cfg)
+    A, Bm = synth.low_rank(cfg)
+    h = B.qllm_build_reassembly(am, theta, W, A, Bm, cfg.w_bits)
+    layer = B.Layer(h, gamma, beta, cfg.ln_eps, None, cfg.a_bits, B.QLLM_BF16, B.QLLM_BF16, max_M=cfg.M)
+    x = synth.activations(cfg)
+    out = torch.zeros((cfg.M, cfg.N), dtype=torch.bfloat16, device=G.DEV)
+    layer.forward(G.dev_x(x), out)
+    torch.cuda.synchronize()
+    assert B.qllm_poll_status() == 0
+    # the oracle on the product's statistic
+    assert oracle.theta_percentile(am, 0.99) == theta
+    ptr, src, coef, st = oracle.build_map(am, theta)
+    p2, s2, c2 = h.map()
+    assert np.array_equal(p2, ptr) and np.array_equal(s2, src) and np.array_equal(c2, coef)
+    w = oracle.prepare_weights(W, ptr, src, cfg.w_bits, A, Bm)
+    wc, ws, wz, wcs = h.weights()
+    assert np.array_equal(wc, oracle.pack4(w["codes"]) if cfg.w_bits == 4 else w["codes"])
+    assert np.array_equal(ws, w["scale"]) and np.array_equal(wz, w["zero"]) and np.array_equal(wcs, w["colsum"])
+    pc, ps, pz, pr, lanes = layer.workspace_ptrs()
+
+    def from_dev(p, shape, typestr):
+        class View:
+            __cuda_array_interface__ = dict(shape=tuple(shape), typestr=typestr, data=(int(p), False), version=2)
+        return torch.as_tensor(View(), device=G.DEV).cpu().numpy().copy()
+
+    codes = from_dev(pc, (cfg.M, cfg.K if lanes == 8 else cfg.K // 2), "|u1")
+    if lanes == 4:
+        codes = parity.unpack_codes(codes, 4)
+    scale, zero, rowsum = from_dev(ps, (cfg.M,), "<f4"), from_dev(pz, (cfg.M,), "<f4"), from_dev(pr, (cfg.M,), "<i4")
+    ref_q = oracle.reassemble_quant(x, gamma, beta, cfg.ln_eps, ptr, src, coef, cfg.a_bits, want_pre=True)
+    parity.check_activation_codes(codes, scale, zero, rowsum, ref_q, cfg.a_bits)
+    acc = oracle.int_matmul(codes, w["codes"])
+    ref = oracle.epilogue(acc, cfg.K, scale, zero, rowsum, w["scale"], w["zero"], w["colsum"], None)
+    parity.check_output(G.bf16_bits(out.cpu()), ref, "bf16")
     layer.destroy()
