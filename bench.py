@@ -227,6 +227,14 @@ def run_gpu(args):
     row = K // 2 if cfg.a_bits == 4 else K
     out = torch.empty((M, N), dtype=out_dtype, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+    flush_r = torch.zeros(256 << 18, dtype=torch.float32, device=dev)
+
+    def flush_l2():
+        # write a buffer larger than L2, then read another one: the cache ends up full of CLEAN lines of data
+        # the step never touches (after the write alone the step's first misses would each pay for the write-back
+        # of a dirty flush line)
+        flush.zero_()
+        flush_r.sum()
 
     MID_EVERY = 2
 
@@ -246,7 +254,7 @@ def run_gpu(args):
 
     sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(args.warmup):
-        flush.zero_()
+        flush_l2()
         step()
     barrier()
     assert B.qllm_poll_status() == 0, "device-side wait timed out during warm-up"
@@ -262,7 +270,7 @@ def run_gpu(args):
         n0 = B.qllm_launch_count()
         barrier()
         for i in range(args.steps):
-            flush.zero_()                  # L2 flush between timed iterations (not inside the event pairs)
+            flush_l2()                     # L2 flush between timed iterations (not inside the event pairs)
             step(events[i], mid=(i % MID_EVERY == 0))
         barrier()
         if rounds == 0:
@@ -347,7 +355,7 @@ def run_gpu(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "u8",
             "data": "synthetic",
             "config": {"workload": f"{cfg.name}: M={M} K={K} N={N} W{cfg.w_bits}A{cfg.a_bits} x=bf16 out=bf16 per GPU",
-                       "l2": "256 MB buffer written between timed iterations", "map_extra_channels": stats["E"],
+                       "l2": "256 MB buffer written, then 256 MB read, between timed iterations", "map_extra_channels": stats["E"],
                        "merged_rows": stats["merged_rows"], "builder_s": round(build_s, 3), "parallelism": f"tokens x{world}"},
             "e2e": {"value": world * M / (ms_e2e_w * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e_w},
@@ -371,6 +379,61 @@ def run_gpu(args):
     layer.destroy()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_fold(args):
+    """Appendix B study: with the reassembly folded into the preceding layer, the run-time stage in front of the GEMM
+    is the per-token quantizer alone (qllm_quantize_rows).  Timed on 16384 token rows of the c2 shape (134 MB in:
+    larger than L2) against the HBM roofline; one launch per step."""
+    import numpy as np
+    import torch
+    from paper_2310_08041_b200 import binding as B
+    from paper_2310_08041_b200 import synth
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    cfg = synth.CONFIGS["c2"].scaled(M=16384)
+    M, K = cfg.M, cfg.K
+    x_np = synth.activations(cfg)
+    x = torch.from_numpy(x_np.view(np.int16)).to(dev).view(torch.bfloat16)
+    codes = torch.empty((M, K // 2), dtype=torch.uint8, device=dev)
+    sc = torch.empty(M, device=dev); ze = torch.empty(M, device=dev); rs = torch.empty(M, dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush_r = torch.zeros(256 << 18, dtype=torch.float32, device=dev)
+
+    def flush_l2():
+        flush.zero_()       # write a buffer larger than L2, then read another: the cache holds clean foreign lines
+        flush_r.sum()
+    sampler = ClockSampler(0)
+    for _ in range(args.warmup):
+        flush_l2()
+        B.qllm_quantize_rows(x, 4, codes, sc, ze, rs)
+    torch.cuda.synchronize()
+    ts = []
+    n0 = B.qllm_launch_count()
+    t_start = time.time()
+    for _ in range(args.steps):
+        flush_l2()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); B.qllm_quantize_rows(x, 4, codes, sc, ze, rs); e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    t_end = time.time()
+    launches = B.qllm_launch_count() - n0
+    clocks = sampler.stop(t_start, t_end)
+    peaks = _peaks()
+    st = _stats(ts)
+    nbytes = M * (K * 2 + K // 2 + 12)
+    gbs = nbytes / (st["median"] * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": M / (st["mean"] * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": st["mean"], "ms_per_step_stats": st, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": f"c2_fold: per-token quantizer alone (Appendix B), M={M} K={K} 4-bit codes, x=bf16",
+                   "l2": "256 MB buffer written, then 256 MB read, between timed iterations; 134 MB of input"},
+        "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": {"kernel": "quantize_rows_warp", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS,
+                     "peak_source": f"{peaks['source']} STREAM-style copy", "bytes": nbytes, "traffic": None}}))
 
 
 def launch_ranks(n, argv):
@@ -416,7 +479,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c2_w4a8"])
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "c5", "c2_w4a8", "c2_fold"])
     ap.add_argument("--ref-rows", type=int, default=0, help="token rows of the oracle sample (0 = auto)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stub", action="store_true",
@@ -433,6 +496,8 @@ def main():
         sys.exit(2)
     if args.stub:
         run_stub(args)
+    elif args.workload == "c2_fold":
+        run_fold(args)
     else:
         run_gpu(args)
 

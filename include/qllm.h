@@ -95,6 +95,15 @@ int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C,
                           int bits, uint8_t* codes, float* a_scale, float* a_zero,
                           int32_t* a_rowsum, void* stream);
 
+/* The per-token quantizer of Eq. 2 alone (device, asynchronous): alpha, zero-point, codes and code sum of every
+ * row of x[M][C], exactly as in qllm_reassemble_quant but with no LayerNorm and no map.  This is the run-time half
+ * of the pre-GEMM stage when the reassembly has been folded into the layer that produces x (Appendix B,
+ * qllm_fold_previous): that layer already emits the reassembled channels.  Arguments, layouts and errors as in
+ * qllm_reassemble_quant.  bf16 rows of up to 8192 channels and fp32 rows of up to 4096 (C a multiple of 256) are
+ * read from memory once. */
+int qllm_quantize_rows(const void* x, int x_dtype, int64_t M, int C, int bits,
+                       uint8_t* codes, float* a_scale, float* a_zero, int32_t* a_rowsum, void* stream);
+
 /* ==========================================================================
  * 2. Low-bit integer GEMM with dequantizing epilogue   (device, asynchronous)
  * ==========================================================================

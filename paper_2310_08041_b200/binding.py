@@ -24,7 +24,7 @@ QLLM_F32, QLLM_BF16 = 0, 1
 
 # every symbol include/qllm.h declares
 EXPORTS = [
-    "qllm_reassemble_quant", "qllm_qgemm", "qllm_qgemm_noalloc", "qllm_qgemm_acc", "qllm_calib_absmax",
+    "qllm_reassemble_quant", "qllm_quantize_rows", "qllm_qgemm", "qllm_qgemm_noalloc", "qllm_qgemm_acc", "qllm_calib_absmax",
     "qllm_build_reassembly", "qllm_build_reassembly_eq5", "qllm_build_reassembly_dist", "qllm_layernorm_rows", "qllm_channel_distance", "qllm_free_reassembly", "qllm_reassembly_map",
     "qllm_reassembly_weights", "qllm_reassembly_stats", "qllm_validate_map", "qllm_fold_previous",
     "qllm_theta_percentile", "qllm_theta_for_extra", "qllm_search_theta",
@@ -42,6 +42,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 _vp, _i, _i64, _f, _d = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_double
 _lib.qllm_reassemble_quant.argtypes = [_vp, _i, _i64, _i, _vp, _vp, _f, _vp, _vp, _vp, _i, _vp, _vp, _vp, _vp, _vp]
+_lib.qllm_quantize_rows.argtypes = [_vp, _i, _i64, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.qllm_qgemm.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.qllm_qgemm_noalloc.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _i, _i, _i, _i, _i, _vp]
 _lib.qllm_qgemm_acc.argtypes = [_vp, _vp, _vp, _i64, _i, _i, _i, _i, _vp]
@@ -126,6 +127,13 @@ def qllm_reassemble_quant(x, ln_gamma, ln_beta, map_ptr, map_src, map_coef, bits
     _check(_lib.qllm_reassemble_quant(_dp(x), _xdtype(x), M, C, _dp(ln_gamma), _dp(ln_beta), ln_eps,
                                       _dp(map_ptr), _dp(map_src), _dp(map_coef), bits, _dp(codes),
                                       _dp(a_scale), _dp(a_zero), _dp(a_rowsum), _stream(stream)))
+
+
+def qllm_quantize_rows(x, bits, codes, a_scale, a_zero, a_rowsum=None, stream=None):
+    """Eq. 2 per token row of x [M][C] (no LayerNorm, no map): the run-time stage of a folded layer (Appendix B)."""
+    M, C = x.shape
+    _check(_lib.qllm_quantize_rows(_dp(x), _xdtype(x), M, C, bits, _dp(codes), _dp(a_scale), _dp(a_zero), _dp(a_rowsum),
+                                   _stream(stream)))
 
 
 def qllm_qgemm(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, bias, out, M, N, K, a_bits, w_bits,

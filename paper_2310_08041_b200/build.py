@@ -12,7 +12,7 @@ OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libqllm_b200.so")
 
 SOURCES = ["api.cu", "builder.cpp", "reassemble_quant.cu", "reassemble_quant_token.cu", "reassemble_quant_generic.cu",
-           "qgemm_plain.cu", "qgemm_decode.cu", "qgemm_tc.cu", "qgemm_tc2.cu", "qgemm_noalloc.cu", "theta_search.cu", "channel_distance.cu", "debug_wait.cu"]
+           "qgemm_plain.cu", "qgemm_decode.cu", "qgemm_tc.cu", "qgemm_tc2.cu", "qgemm_noalloc.cu", "theta_search.cu", "channel_distance.cu", "debug_wait.cu", "quantize_rows.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-ffp-contract=off", "--expt-relaxed-constexpr"]

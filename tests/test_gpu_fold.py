@@ -39,3 +39,39 @@ def test_fold_previous_matches_oracle_and_quantizes_without_layernorm():
             parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref, bits)
         finally:
             parity.FLIP_BAND = old
+
+
+@pytest.mark.parametrize("M,C,dtype,bits", [(40, 256, "f32", 4), (33, 4096, "bf16", 4), (19, 5120, "bf16", 6),
+                                            (9, 8192, "bf16", 8), (21, 250, "f32", 6), (5, 77, "bf16", 8),
+                                            (3, 4096, "f32", 4)])
+def test_quantize_rows_alone(M, C, dtype, bits):
+    """The run-time stage of a folded layer through its own entry point: Eq. 2 per row, no LayerNorm, no map,
+    against the oracle's quantizer on the same values (constant and all-zero rows included)."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    rng = np.random.default_rng(C + bits)
+    x = (rng.standard_normal((M, C)) * (1 + 25 * (rng.random(C) < 0.02))).astype(np.float32)
+    x[0] = 0.0
+    if M > 2:
+        x[2] = -3.25
+    if dtype == "bf16":
+        xb = synth.f32_to_bf16_bits(x)
+        x64 = synth.bf16_bits_to_f32(xb).astype(np.float64)
+        xd = G.dev_x(xb)
+    else:
+        x64 = x.astype(np.float64)
+        xd = G.dev(x)
+    codes = torch.full((M, C // 2 if bits == 4 else C), 0xAB, dtype=torch.uint8, device=G.DEV)
+    sc = torch.zeros(M, device=G.DEV); ze = torch.zeros(M, device=G.DEV); rs = torch.zeros(M, dtype=torch.int32, device=G.DEV)
+    B.qllm_quantize_rows(xd, bits, codes, sc, ze, rs)
+    torch.cuda.synchronize()
+    got = codes.cpu().numpy()
+    got = parity.unpack_codes(got, 4) if bits == 4 else got
+    ref = oracle.quant_rows(x64, bits, want_pre=True)
+    old = parity.FLIP_BAND
+    parity.FLIP_BAND = old * (17 if bits == 8 else 1)
+    try:
+        parity.check_activation_codes(got, sc.cpu().numpy(), ze.cpu().numpy(), rs.cpu().numpy(), ref, bits)
+    finally:
+        parity.FLIP_BAND = old
