@@ -157,7 +157,8 @@ bool expand_path(int64_t M, int N, int K, int a_bits, int w_bits) {
 // w_ready: the weight codes already expanded to bytes at the weight slot of this stream's expand scratch
 // (done ahead of time on another stream by the layer object), or nullptr.
 int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
-                  const EpilogueArgs& ep, cudaStream_t st, bool may_allocate, const uint8_t* w_ready = nullptr) {
+                  const EpilogueArgs& ep, cudaStream_t st, bool may_allocate, const uint8_t* w_ready = nullptr,
+                  bool weights_static = false) {
     if (M == 0) return QLLM_OK;
     if (M <= 16 && qgemm_decode_supported(M, N, K, a_bits, w_bits))
         return launch_qgemm_decode(a, w, M, N, K, a_bits, w_bits, ep, st);
@@ -177,7 +178,7 @@ int dispatch_gemm(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, i
             if (writes) { rc = scratch_write_end(kScratchExpand, st, st, nullptr); if (rc != QLLM_OK) return rc; }
             return launch_qgemm_tc(a, w, M, N, K, 8, 8, ep, st);
         }
-        return launch_qgemm_tc(a, w, M, N, K, a_bits, w_bits, ep, st);
+        return launch_qgemm_tc(a, w, M, N, K, a_bits, w_bits, ep, st, weights_static);
     }
     return launch_qgemm_plain(a, w, M, N, K, a_bits, w_bits, ep, st);
 }
@@ -201,7 +202,7 @@ int gemm_check_args(const uint8_t* codes, const float* a_scale, const float* a_z
 int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
                const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
                int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
-               cudaStream_t st, bool may_allocate, const uint8_t* w_ready) {
+               cudaStream_t st, bool may_allocate, const uint8_t* w_ready, bool weights_static) {
     int rc = gemm_check_args(codes, a_scale, a_zero, w_codes, w_scale, w_zero, w_colsum, out, M, N, K, a_bits, w_bits,
                              out_dtype);
     if (rc != QLLM_OK) return rc;
@@ -216,7 +217,7 @@ int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, 
         a_rowsum = scratch;
     }
     EpilogueArgs ep{a_scale, a_zero, a_rowsum, w_scale, w_zero, w_colsum, bias, out, out_dtype, 0};
-    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, st, may_allocate, w_ready);
+    return dispatch_gemm(codes, w_codes, M, N, K, a_bits, w_bits, ep, st, may_allocate, w_ready, weights_static);
 }
 
 }  // namespace qllm
@@ -455,7 +456,7 @@ int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {
     L->w_ready = nullptr;
     return gemm_entry(L->codes, L->a_scale, L->a_zero, L->w_codes, L->w_scale, L->w_zero, L->w_colsum, L->bias,
                       out, M, L->N, L->C, L->lane_bits == 8 ? 8 : L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum,
-                      static_cast<cudaStream_t>(stream), true, w_ready);
+                      static_cast<cudaStream_t>(stream), true, w_ready, true);   // the layer's weights are written by no kernel
 }
 
 int qllm_layer_forward(qllm_layer_t* L, const void* x, int64_t M, void* out, void* stream) {

@@ -133,7 +133,7 @@ int launch_expand_codes(const uint8_t* packed, int64_t rows, int K, uint8_t* byt
 int gemm_entry(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
                const float* w_scale, const float* w_zero, const int32_t* w_colsum, const float* bias, void* out,
                int64_t M, int N, int K, int a_bits, int w_bits, int out_dtype, const int32_t* a_rowsum,
-               cudaStream_t st, bool may_allocate, const uint8_t* w_ready = nullptr);
+               cudaStream_t st, bool may_allocate, const uint8_t* w_ready = nullptr, bool weights_static = false);
 int gemm_check_args(const uint8_t* codes, const float* a_scale, const float* a_zero, const uint8_t* w_codes,
                     const float* w_scale, const float* w_zero, const int32_t* w_colsum, const void* out, int64_t M,
                     int N, int K, int a_bits, int w_bits, int out_dtype);
@@ -147,8 +147,10 @@ bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits);
 bool qgemm_tc2_supported(int64_t M, int N, int K, int a_bits, int w_bits);
 int launch_qgemm_tc2(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const EpilogueArgs& ep,
                      cudaStream_t st);
+// weights_static: the caller vouches that no kernel before this one on the stream writes the weights (they may then
+// be requested before that kernel is complete)
 int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits,
-                    int w_bits, const EpilogueArgs& ep, cudaStream_t st);
+                    int w_bits, const EpilogueArgs& ep, cudaStream_t st, bool weights_static = false);
 bool qgemm_decode_supported(int64_t M, int N, int K, int a_bits, int w_bits);
 
 }  // namespace qllm

@@ -45,7 +45,7 @@ struct Tile {
 template <int BN, bool AP, bool WP>
 __global__ void __launch_bounds__(Tile<BN, AP, WP>::THREADS, 1)
 qgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
-                int64_t M, int N, int K, EpilogueArgs ep, int* status, uint32_t opa_tx) {
+                int64_t M, int N, int K, EpilogueArgs ep, int* status, uint32_t opa_tx, int early_w) {
     using T = Tile<BN, AP, WP>;
     constexpr int S = T::STAGES;
     extern __shared__ uint8_t smem_dyn[];
@@ -97,26 +97,44 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
     // The kernel is launched as a programmatic dependent of the kernel before it on the stream (for a layer, the
     // pre-GEMM kernel that writes the tokens): everything above touched no global memory and has run under that
-    // kernel and the launch latency; nothing below starts before that kernel is complete.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // kernel and the launch latency.  Every role that touches global memory waits for that kernel to be complete
+    // (griddepcontrol.wait) before it does; with early_w (the caller vouches that no kernel before this one on the
+    // stream writes the weights: a layer's own weights) the producer first asks for the weight tiles of its first
+    // stages, so that they travel while the tokens are still being written.
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, pre = 0;
             bool ok = true;
+            if (early_w && int(blockIdx.x) < num_tiles) {
+                // the first stages of the first tile: barriers armed for both operands, weight copies on their way
+                const int n0 = (int(blockIdx.x) / tiles_m) * BN;
+                pre = uint32_t(KB < S ? KB : S);
+                for (uint32_t kb = 0; kb < pre; ++kb) {
+                    if (AP || WP) ptx::mbar_arrive_expect_tx(&full_raw[kb], T::RAWA + T::RAWW);
+                    if (!AP || !WP) ptx::mbar_arrive_expect_tx(&full_op[kb], (AP ? 0 : opa_tx) + (WP ? 0 : T::OPW));
+                    if (WP) ptx::tma_load_2d(rawW + kb * T::RAWW, &tmW, int(kb) * (BK / 2), n0, &full_raw[kb]);
+                    else    ptx::tma_load_2d(opW + kb * T::OPW, &tmW, int(kb) * BK, n0, &full_op[kb]);
+                }
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1;
-                    if (!wait_bounded(&empty[s], ph ^ 1, ab)) { ok = false; break; }
-                    if (AP || WP) ptx::mbar_arrive_expect_tx(&full_raw[s], T::RAWA + T::RAWW);
-                    if (!AP || !WP) ptx::mbar_arrive_expect_tx(&full_op[s], (AP ? 0 : opa_tx) + (WP ? 0 : T::OPW));
+                    if (it >= pre) {
+                        if (!wait_bounded(&empty[s], ph ^ 1, ab)) { ok = false; break; }
+                        if (AP || WP) ptx::mbar_arrive_expect_tx(&full_raw[s], T::RAWA + T::RAWW);
+                        if (!AP || !WP) ptx::mbar_arrive_expect_tx(&full_op[s], (AP ? 0 : opa_tx) + (WP ? 0 : T::OPW));
+                    }
                     if (AP) ptx::tma_load_2d(rawA + s * T::RAWA, &tmA, kb * (BK / 2), m0, &full_raw[s]);
                     else    ptx::tma_load_2d(opA + s * T::OPA, &tmA, kb * BK, m0, &full_op[s]);
-                    if (WP) ptx::tma_load_2d(rawW + s * T::RAWW, &tmW, kb * (BK / 2), n0, &full_raw[s]);
-                    else    ptx::tma_load_2d(opW + s * T::OPW, &tmW, kb * BK, n0, &full_op[s]);
+                    if (it >= pre) {
+                        if (WP) ptx::tma_load_2d(rawW + s * T::RAWW, &tmW, kb * (BK / 2), n0, &full_raw[s]);
+                        else    ptx::tma_load_2d(opW + s * T::OPW, &tmW, kb * BK, n0, &full_op[s]);
+                    }
                 }
             }
             if (!ok) {
@@ -162,6 +180,7 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int quad = warp & 3;                        // TMEM lanes 32*quad .. +31
         const int et = threadIdx.x - 32 * kFirstEpiWarp;  // 0..127
         uint32_t lt = 0;
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // the row terms below come from the kernel before
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++lt) {
             const uint32_t abuf = lt & 1, aph = (lt >> 1) & 1;
             const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
@@ -217,7 +236,8 @@ qgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }
 
 template <int BN, bool AP, bool WP>
-int launch(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const EpilogueArgs& ep, cudaStream_t st) {
+int launch(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const EpilogueArgs& ep, cudaStream_t st,
+           bool early_w) {
     using T = Tile<BN, AP, WP>;
     static_assert(T::STAGES >= 2, "pipeline needs at least two stages");
     CUtensorMap tmA, tmW;
@@ -238,7 +258,7 @@ int launch(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, const Ep
     const int64_t tiles = ((M + BM - 1) / BM) * int64_t((N + BN - 1) / BN);
     const int grid = int(std::min<int64_t>(tiles, device_sm_count()));
     QLLM_CUDA_TRY(launch_dependent(kern, dim3(grid), dim3(T::THREADS), T::SMEM, st, tmA, tmW, M, N, K, ep, status,
-                                   uint32_t(a_rows * BK)));
+                                   uint32_t(a_rows * BK), early_w ? 1 : 0));
     return after_launch();
 }
 
@@ -250,7 +270,7 @@ bool qgemm_tc_supported(int64_t M, int N, int K, int a_bits, int w_bits) {
 }
 
 int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, int a_bits, int w_bits,
-                    const EpilogueArgs& ep, cudaStream_t st) {
+                    const EpilogueArgs& ep, cudaStream_t st, bool weights_static) {
     const bool ap = a_bits == 4, wp = w_bits == 4;
     if (!ap && !wp && qgemm_tc2_supported(M, N, K, a_bits, w_bits)) return launch_qgemm_tc2(a, w, M, N, K, ep, st);
     // Tile width by estimated time: rounds of tiles over the SMs x what one tile costs per unit of K.  Byte-lane
@@ -265,7 +285,7 @@ int launch_qgemm_tc(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K,
     int best = 256;
     for (int bn : {192, 160, 128, 96, 64})
         if (cost(bn) < cost(best)) best = bn;
-#define QLLM_TC(BN_, AP_, WP_) launch<BN_, AP_, WP_>(a, w, M, N, K, ep, st)
+#define QLLM_TC(BN_, AP_, WP_) launch<BN_, AP_, WP_>(a, w, M, N, K, ep, st, weights_static)
 #define QLLM_TC_BN(AP_, WP_) \
     (best == 256 ? QLLM_TC(256, AP_, WP_) : best == 192 ? QLLM_TC(192, AP_, WP_) : best == 160 ? QLLM_TC(160, AP_, WP_) : \
      best == 128 ? QLLM_TC(128, AP_, WP_) : best == 96 ? QLLM_TC(96, AP_, WP_) : QLLM_TC(64, AP_, WP_))
