@@ -24,6 +24,20 @@
  * w_codes, out) must be 16-byte aligned (QLLM_ERR_ALIGN otherwise).  There is
  * no CPU fallback: without a usable CUDA device the device calls fail with
  * QLLM_ERR_CUDA.
+ *
+ * DEVICE MEMORY.  Which calls may call cudaMalloc / cudaFree:
+ *   never      qllm_qgemm_noalloc, qllm_quantize_rows, qllm_calib_absmax, qllm_layernorm_rows,
+ *              qllm_channel_distance, qllm_layer_forward / _reassemble_quant / _qgemm / _forward_host (everything a
+ *              layer needs is taken in qllm_layer_create and returned in qllm_layer_destroy);
+ *   grow-only  qllm_reassemble_quant (compiled-map scratch per (device, stream): grown on the first call
+ *              and when C grows), qllm_qgemm and qllm_qgemm_acc (row-sum scratch when a_rowsum = NULL;
+ *              widened-code scratch for a 4-bit operand at M >= 385): library-owned buffers, sized by the
+ *              largest call so far, kept until the process exits;
+ *   always     the offline calls qllm_build_reassembly_eq5 and qllm_search_theta (take and return what
+ *              they need inside the call), qllm_layer_create and qllm_layer_keep_byte_weights.
+ * qllm_layer_forward_host takes no memory either (its device staging comes from qllm_layer_create); its first
+ * chunked call creates two streams and a few events, which the layer keeps.
+ * A grow-only call that found its scratch large enough launches kernels only.
  */
 #ifndef QLLM_H_
 #define QLLM_H_
@@ -88,6 +102,20 @@ extern "C" {
  *  a_zero    device out float[M]  (zero-point, integer-valued)
  *  a_rowsum  device out int32[M] or NULL: sum_c q_c, needed by the GEMM epilogue
  *  M = 0 is a successful no-op.  C <= 49152 (the normalised row is held in shared memory).
+ *
+ *  Cost of the direct call.  The kernel reads the map in a compiled form (per-source weights, gather positions,
+ *  records of the merged rows).  This call receives plain CSR arrays that it may not keep and whose contents the
+ *  caller may change between calls.  It therefore keeps the compiled form of the last map used on `stream` in
+ *  scratch the library owns per (device, stream), beside a 64-bit hash of everything the form depends on (C, the
+ *  three map arrays, ln_gamma, ln_beta: contents, not addresses).  Every call launches one single-CTA kernel ahead
+ *  of the main one that hashes the arrays it was given and recompiles only when the hash differs from the one
+ *  kept (two different contents share a hash with probability 2^-64).  Bf16 rows of 4096 / 5120 / 8192 channels:
+ *  the call also launches the shape-agnostic kernel behind the main one, which returns at once unless the map
+ *  is one the main kernel declines (a source channel read with different coefficients: no product of Eq. 3 /
+ *  Eq. 4, but a legal argument).  Measured at M = 2048, C = 4096 with a cold L2: 49 us per call with the map
+ *  unchanged, 60 us when it is recompiled, against 27 us for the same kernel launched by a layer object
+ *  (section 5), which compiles its map once in qllm_layer_create and knows its sizes: use a layer wherever the
+ *  map is fixed.
  */
 int qllm_reassemble_quant(const void* x, int x_dtype, int64_t M, int C,
                           const float* ln_gamma, const float* ln_beta, float ln_eps,
@@ -320,6 +348,14 @@ int qllm_layer_forward(qllm_layer_t* layer, const void* x, int64_t M, void* out,
  * layer's weights into out[M][N] (device).  Asynchronous on stream. */
 int qllm_layer_reassemble_quant(qllm_layer_t* layer, const void* x, int64_t M, void* stream);
 int qllm_layer_qgemm(qllm_layer_t* layer, int64_t M, void* out, void* stream);
+/* Memory for time, opt-in: keep != 0 gives a layer with 4-bit weights a second, resident copy of them with one
+ * code per byte (N * C bytes of device memory; cudaMalloc + one kernel on stream, the call waits for it).  Calls
+ * of 385 tokens and more then skip the per-call widening of the weights (a read of N*C/2 and a write of N*C bytes
+ * that runs beside the pre-GEMM kernel: 13-17 us of a 95 us step at M = 2048, C = 4096, N = 12288), calls of 17 to
+ * 384 tokens read byte tiles instead of unpacking 4-bit tiles in shared memory (2-3 us of 35); the decode path
+ * (M <= 16) keeps streaming the 4-bit codes.  Results are bit-identical either way.  keep = 0 waits for
+ * stream and frees the copy.  Not to be called while a forward of this layer is being issued from another thread. */
+int qllm_layer_keep_byte_weights(qllm_layer_t* layer, int keep, void* stream);
 /* x, out: HOST (pinned memory makes the copies asynchronous).  Copies x to the device, runs the
  * path, copies out back and waits until all of it is done.  Calls of 2048 tokens or more are cut into four
  * chunks of token rows whose copy in, kernels and copy out overlap on two internal copy streams (the host link

@@ -30,7 +30,7 @@ EXPORTS = [
     "qllm_theta_percentile", "qllm_theta_for_extra", "qllm_search_theta",
     "qllm_layer_create", "qllm_layer_destroy", "qllm_layer_forward", "qllm_layer_forward_host",
     "qllm_layer_reassemble_quant", "qllm_layer_qgemm",
-    "qllm_layer_workspace",
+    "qllm_layer_workspace", "qllm_layer_keep_byte_weights",
     "qllm_status_string", "qllm_last_cuda_error", "qllm_poll_status", "qllm_launch_count", "qllm_debug_wait_expiry",
 ]
 
@@ -74,6 +74,7 @@ _lib.qllm_layer_reassemble_quant.argtypes = [_vp, _vp, _i64, _vp]
 _lib.qllm_layer_qgemm.argtypes = [_vp, _i64, _vp, _vp]
 _lib.qllm_layer_workspace.argtypes = [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_vp),
                                       ctypes.POINTER(ctypes.c_int)]
+_lib.qllm_layer_keep_byte_weights.argtypes = [_vp, _i, _vp]
 _lib.qllm_status_string.argtypes = [_i]
 _lib.qllm_status_string.restype = ctypes.c_char_p
 _lib.qllm_launch_count.restype = _i64
@@ -354,6 +355,9 @@ class Layer:
 
     def qgemm(self, M, out, stream=None):
         _check(_lib.qllm_layer_qgemm(self._h, M, _dp(out), _stream(stream)))
+
+    def keep_byte_weights(self, keep=True, stream=None):
+        _check(_lib.qllm_layer_keep_byte_weights(self._h, 1 if keep else 0, _stream(stream)))
 
     def forward_host(self, x_host, out_host, M, stream=None):
         """x_host/out_host: host pointers (ints) or numpy arrays / pinned CPU torch tensors."""

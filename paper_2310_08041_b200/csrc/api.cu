@@ -103,6 +103,7 @@ int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out) {
         QLLM_CUDA_TRY(cudaMalloc(&e->ptr, bytes));
         e->cap = bytes;
         ++e->epoch;
+        if (kind == kScratchMapImage) QLLM_CUDA_TRY(cudaMemsetAsync(e->ptr, 0, std::min(bytes, kMapScratchHeader), st));
     }
     *out = e->ptr;
     return QLLM_OK;
@@ -253,6 +254,9 @@ struct qllm_layer {
     // 4-bit activations of a call that will take the byte-lane GEMM are written one code per byte by the
     // pre-GEMM kernel itself (no expansion pass): lane width of the codes now in the workspace
     int lane_bits = 0;
+    // optional resident copy of the 4-bit weights, one code per byte (qllm_layer_keep_byte_weights): large-M calls
+    // then widen nothing per call
+    uint8_t* w_wide = nullptr;
     std::vector<void*> owned;
 };
 
@@ -401,6 +405,7 @@ void qllm_layer_destroy(qllm_layer_t* L) {
     for (cudaEvent_t e : L->ev_in) if (e) cudaEventDestroy(e);
     for (cudaEvent_t e : L->ev_done) if (e) cudaEventDestroy(e);
     for (void* p : L->owned) cudaFree(p);
+    if (L->w_wide) cudaFree(L->w_wide);
     delete L;
 }
 
@@ -408,7 +413,7 @@ int qllm_layer_reassemble_quant(qllm_layer_t* L, const void* x, int64_t M, void*
     if (!L || !x) return QLLM_ERR_NULL;
     if (M < 0 || M > L->max_M) return QLLM_ERR_SHAPE;
     L->w_ready = nullptr;
-    const bool expand = expand_path(M, L->N, L->C, L->a_bits, L->w_bits);
+    const bool expand = !L->w_wide && expand_path(M, L->N, L->C, L->a_bits, L->w_bits);
     // 4-bit activations for a tensor-core GEMM (more than 16 tokens) are written one code per byte: the GEMM
     // then expands nothing on the activation side (below kExpandMinM tokens it unpacks only its weight tiles)
     const bool byte_lanes = L->a_bits == 4 && M > 16 && qgemm_tc_supported(M, L->N, L->C, L->a_bits, L->w_bits) &&
@@ -454,9 +459,42 @@ int qllm_layer_qgemm(qllm_layer_t* L, int64_t M, void* out, void* stream) {
         w_ready = L->w_ready;
     }
     L->w_ready = nullptr;
+    const int a_lane = L->lane_bits == 8 ? 8 : L->a_bits;
+    // the resident byte copy serves every tensor-core call (same codes in 8-bit lanes: nothing is widened per call
+    // from 385 tokens, no weight tile is unpacked in shared memory below); decode keeps streaming the 4-bit codes
+    if (L->w_wide && M > 16 && qgemm_tc_supported(M, L->N, L->C, a_lane, 8))
+        return gemm_entry(L->codes, L->a_scale, L->a_zero, L->w_wide, L->w_scale, L->w_zero, L->w_colsum, L->bias, out, M,
+                          L->N, L->C, a_lane, 8, L->out_dtype, L->a_rowsum, static_cast<cudaStream_t>(stream), true,
+                          nullptr, true);
     return gemm_entry(L->codes, L->a_scale, L->a_zero, L->w_codes, L->w_scale, L->w_zero, L->w_colsum, L->bias,
-                      out, M, L->N, L->C, L->lane_bits == 8 ? 8 : L->a_bits, L->w_bits, L->out_dtype, L->a_rowsum,
+                      out, M, L->N, L->C, a_lane, L->w_bits, L->out_dtype, L->a_rowsum,
                       static_cast<cudaStream_t>(stream), true, w_ready, true);   // the layer's weights are written by no kernel
+}
+
+int qllm_layer_keep_byte_weights(qllm_layer_t* L, int keep, void* stream) {
+    if (!L) return QLLM_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!keep) {
+        if (L->w_wide) {
+            QLLM_CUDA_TRY(cudaStreamSynchronize(st));             // a GEMM of this layer may still be reading it
+            if (L->side) QLLM_CUDA_TRY(cudaStreamSynchronize(L->side));
+            QLLM_CUDA_TRY(cudaFree(L->w_wide));
+            L->w_wide = nullptr;
+        }
+        return QLLM_OK;
+    }
+    if (L->w_bits != 4 || L->w_wide) return QLLM_OK;              // nothing to widen / already there
+    void* p = nullptr;
+    if (cudaMalloc(&p, size_t(L->N) * size_t(L->C)) != cudaSuccess) { cudaGetLastError(); return QLLM_ERR_NOMEM; }
+    int rc = launch_expand_codes(L->w_codes, L->N, L->C, static_cast<uint8_t*>(p), st);
+    if (rc == QLLM_OK) {
+        const cudaError_t e = cudaStreamSynchronize(st);
+        if (e != cudaSuccess) rc = cuda_fail(e);
+    }
+    if (rc != QLLM_OK) { cudaFree(p); return rc; }
+    L->w_wide = static_cast<uint8_t*>(p);
+    L->w_ready = nullptr;
+    return QLLM_OK;
 }
 
 int qllm_layer_forward(qllm_layer_t* L, const void* x, int64_t M, void* out, void* stream) {

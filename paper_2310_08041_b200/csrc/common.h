@@ -81,7 +81,10 @@ struct EpilogueArgs {
 };
 
 // Per-(device, stream) library scratch, grown on demand and never shrunk.
+// The map-image scratch starts with a header of kMapScratchHeader bytes whose first 8 hold the content key of the
+// token-kernel image behind it (0 = none; a fresh allocation is zeroed on the stream).
 enum ScratchKind { kScratchExpand = 0, kScratchMapImage = 1, kScratchKinds = 2 };
+constexpr size_t kMapScratchHeader = 256;
 int stream_scratch(int kind, cudaStream_t st, size_t bytes, uint8_t** out);
 
 // The specialised fused kernels consume a compiled image of the reassembly map (0 bytes: the channel
@@ -106,8 +109,10 @@ int reassemble_map_counts(int C, int x_dtype, const void* image, cudaStream_t st
 // The kernel for bf16 rows of LLaMA hidden sizes (reassemble_quant_token.cu)
 bool token_kernel_serves(int C);
 size_t token_image_bytes(int C);
+// key (device, may be null): content key kept beside an image in library scratch; when the inputs hash to the
+// value found there the image is left as it is
 int compile_token_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
-                      const float* coef, void* image, cudaStream_t st);
+                      const float* coef, void* image, cudaStream_t st, uint64_t* key = nullptr);
 int token_map_counts(int C, const void* image, cudaStream_t st, MapCounts* out);
 // device word of a compiled token image: non-zero when the token kernel serves the map
 const int* token_image_served_flag(int C, const void* image);

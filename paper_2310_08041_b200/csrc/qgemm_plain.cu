@@ -106,7 +106,7 @@ expand_codes_kernel(const uint4* __restrict__ packed, int64_t chunks, uint4* __r
 int launch_expand_codes(const uint8_t* packed, int64_t rows, int K, uint8_t* bytes, cudaStream_t st) {
     const int64_t chunks = rows * (K / 32);
     if (chunks == 0) return QLLM_OK;
-    const int grid = int(std::min<int64_t>((chunks + 255) / 256, 148 * 16));
+    const int grid = int(std::min<int64_t>((chunks + 255) / 256, int64_t(device_sm_count()) * 16));
     expand_codes_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const uint4*>(packed), chunks,
                                               reinterpret_cast<uint4*>(bytes));
     return after_launch();

@@ -504,13 +504,18 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
     if (map_image && counts) mc = *counts;
     if (token_path(C, x_dtype)) {
         if (!map_image) {
-            // direct call: the map is compiled for this launch into per-stream library scratch (one launch); the
-            // token kernel serves it if the image says it can, else the shape-agnostic kernel behind it does
+            // direct call: the map is compiled into per-stream library scratch by one launch ahead of the kernel,
+            // which first hashes the map, gamma and beta and leaves the image alone when it was made from the
+            // same contents (the key sits at the start of the scratch; whatever else writes the scratch resets
+            // it); the token kernel serves the image if the image says it can, else the shape-agnostic kernel
+            // behind it does
             uint8_t* buf = nullptr;
-            int rc = stream_scratch(kScratchMapImage, st, token_image_bytes(C), &buf);
+            int rc = stream_scratch(kScratchMapImage, st, kMapScratchHeader + token_image_bytes(C), &buf);
             if (rc != QLLM_OK) return rc;
-            rc = compile_token_map(C, gamma, beta, ptr, src, coef, buf, st);
+            rc = compile_token_map(C, gamma, beta, ptr, src, coef, buf + kMapScratchHeader, st,
+                                   reinterpret_cast<uint64_t*>(buf));
             if (rc != QLLM_OK) return rc;
+            buf += kMapScratchHeader;
             rc = launch_reassemble_quant_token(x, M, C, gamma, beta, eps, ptr, src, coef, bits, buf, MapCounts(), codes,
                                                a_scale, a_zero, a_rowsum, st, false, share_sm);
             if (rc != QLLM_OK) return rc;
@@ -527,8 +532,10 @@ int launch_reassemble_quant(const void* x, int x_dtype, int64_t M, int C, const 
     if (!map_image) {
         // direct call: compile the map for this launch into per-stream library scratch
         uint8_t* buf = nullptr;
-        int rc = stream_scratch(kScratchMapImage, st, warp_image_bytes(C), &buf);
+        int rc = stream_scratch(kScratchMapImage, st, kMapScratchHeader + warp_image_bytes(C), &buf);
         if (rc != QLLM_OK) return rc;
+        QLLM_CUDA_TRY(cudaMemsetAsync(buf, 0, 16, st));     // no token-kernel image is in the scratch any more
+        buf += kMapScratchHeader;
         rc = compile_warp_map(C, gamma, beta, ptr, src, coef, buf, st);
         if (rc != QLLM_OK) return rc;
         map_image = buf;

@@ -43,14 +43,55 @@ __device__ __forceinline__ void put_source(const TokImage& im, int k, float w, f
     (((k & 7) < 4) ? im.bsA : im.bsB)[4 * (k >> 3) + (k & 3)] = b;
 }
 
+// 64-bit finaliser of the splitmix64 generator (Steele, Lea, Flood 2014): every input bit reaches every output bit
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+// Content key of everything a compiled image depends on: the sum over all elements of mix64(array, index, bits),
+// plus the sizes.  Order-independent, so every thread adds up a strided share.  Never 0 (0 marks "no image").
+__device__ uint64_t map_content_key(int C, const float* gamma, const float* beta, const int32_t* ptr,
+                                    const int32_t* src, const float* coef, uint64_t* red) {
+    const int nnz = __ldg(ptr + C);
+    uint64_t h = 0;
+    auto add = [&](uint64_t array, int i, uint32_t bits) { h += mix64((array << 56) ^ (uint64_t(uint32_t(i)) << 32) ^ bits); };
+    for (int i = threadIdx.x; i <= C; i += blockDim.x) add(1, i, uint32_t(__ldg(ptr + i)));
+    for (int i = threadIdx.x; i < nnz; i += blockDim.x) {
+        add(2, i, uint32_t(__ldg(src + i)));
+        add(3, i, __float_as_uint(__ldg(coef + i)));
+    }
+    for (int i = threadIdx.x; i < C; i += blockDim.x) {
+        add(4, i, __float_as_uint(__ldg(gamma + i)));
+        if (beta) add(5, i, __float_as_uint(__ldg(beta + i)));
+    }
+    for (int o = 16; o > 0; o >>= 1) h += __shfl_xor_sync(0xffffffffu, h, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = h;
+    __syncthreads();
+    h = mix64((uint64_t(uint32_t(C)) << 32) ^ uint32_t(nnz) ^ (beta ? 1ull << 63 : 0ull));
+    for (int w = 0; w < int(blockDim.x >> 5); ++w) h += red[w];
+    return h ? h : 1;
+}
+
 // One CTA compiles the whole map: a counting pass, then one thread per output channel writes its record, the
 // weights of the sources it reads and, for a multi-entry row, its slot.
+// key (may be null): where the content key of the image's inputs is kept beside an image that lives in library
+// scratch.  A call whose inputs hash to the key already there finds its image in place and compiles nothing.
 __global__ void __launch_bounds__(1024)
 compile_map_token_kernel(int C, const float* __restrict__ gamma, const float* __restrict__ beta,
                          const int32_t* __restrict__ ptr, const int32_t* __restrict__ src,
-                         const float* __restrict__ coef, TokImage im) {
+                         const float* __restrict__ coef, TokImage im, uint64_t* key) {
     __shared__ int cnt[8];
+    __shared__ uint64_t red[32];
     constexpr uint32_t kUnread = 0xFFFFFFFFu;
+    uint64_t content = 0;
+    if (key) {
+        content = map_content_key(C, gamma, beta, ptr, src, coef, red);
+        if (*key == content) return;                          // the same value for every thread
+        __syncthreads();
+        if (threadIdx.x == 0) *key = 0;                       // no valid image while this one is being written
+    }
     if (threadIdx.x < 8) cnt[threadIdx.x] = 0;
     for (int i = threadIdx.x; i < C / 32; i += blockDim.x) im.member[i] = 0u;
     for (int k = threadIdx.x; k < C; k += blockDim.x) { im.tag[k] = kUnread; im.nmulti[k] = 0; }
@@ -128,6 +169,7 @@ compile_map_token_kernel(int C, const float* __restrict__ gamma, const float* __
     }
     __syncthreads();
     if (threadIdx.x < 8) im.head[threadIdx.x] = threadIdx.x == 7 ? int(fits && cnt[7] == 0) : cnt[threadIdx.x];
+    if (key && threadIdx.x == 0) { __threadfence(); *key = content; }
 }
 
 // Output channel c from the stored row y by its CSR row: y[src] for a single entry (the coefficient is in y
@@ -663,9 +705,9 @@ bool token_kernel_serves(int C) { return C == 4096 || C == 5120 || C == 8192; }
 size_t token_image_bytes(int C) { return token_kernel_serves(C) ? (tok_image_bytes_impl(C) + 15) / 16 * 16 : 0; }
 
 int compile_token_map(int C, const float* gamma, const float* beta, const int32_t* ptr, const int32_t* src,
-                      const float* coef, void* image, cudaStream_t st) {
+                      const float* coef, void* image, cudaStream_t st, uint64_t* key) {
     if (!token_kernel_serves(C)) return QLLM_ERR_UNSUPPORTED;
-    compile_map_token_kernel<<<1, 1024, 0, st>>>(C, gamma, beta, ptr, src, coef, tok_image_at(image, C));
+    compile_map_token_kernel<<<1, 1024, 0, st>>>(C, gamma, beta, ptr, src, coef, tok_image_at(image, C), key);
     return after_launch();
 }
 

@@ -69,6 +69,13 @@ def test_layer_forward_matches_oracle(name, kw, out_dtype):
     oh = torch.zeros((cfg.M, cfg.N), dtype=tdt).pin_memory()
     layer.forward_host(xh, oh, cfg.M)
     assert torch.equal(oh.view(torch.int16 if out_dtype == "bf16" else torch.int32), o.view(torch.int16 if out_dtype == "bf16" else torch.int32))
+    # the resident byte copy of 4-bit weights changes which kernel variant runs, not a bit of the result
+    layer.keep_byte_weights(True)
+    out2 = torch.zeros_like(out)
+    layer.forward(G.dev_x(x), out2)
+    torch.cuda.synchronize()
+    assert torch.equal(out2, out)
+    layer.keep_byte_weights(False)
     # informational: the quantized layer approximates the fp64 layer
     y = oracle.layernorm(x, L["gamma"], L["beta"], cfg.ln_eps)
     dense = oracle.dense_linear(y, L["W"].astype(np.float64)) + bias
@@ -144,6 +151,25 @@ def test_layer_full_size_two_halves_sampled(name):
     diff = oh.view(torch.int16) != out.cpu().view(torch.int16)
     assert not bool(diff.any()), (f"{int(diff.sum())} entries differ, rows {torch.nonzero(diff.any(1)).flatten()[:8].tolist()}"
                                   f" cols {torch.nonzero(diff.any(0)).flatten()[:8].tolist()}")
+    # with the resident byte copy of the weights (no per-call widening) the step returns the same bytes, on both
+    # entry points, and so does the layer after the copy has been given back
+    want = out.cpu().view(torch.int16).clone()
+    layer.keep_byte_weights(True)
+    for step in ("resident", "resident-host", "released"):
+        out.zero_()
+        if step == "resident-host":
+            oh.zero_()
+            layer.forward_host(xh, oh, M)
+            got = oh.view(torch.int16)
+        else:
+            if step == "released":
+                layer.keep_byte_weights(False)
+            layer.reassemble_quant(xd)
+            layer.qgemm(M, out)
+            torch.cuda.synchronize()
+            got = out.cpu().view(torch.int16)
+        assert torch.equal(got, want), step
+    assert B.qllm_poll_status() == 0
     layer.destroy()
 
 

@@ -211,3 +211,67 @@ def test_handmade_maps_on_the_token_kernel_shapes(kind, C):
         got = G.run_reassemble_quant(x, g, None, 1e-5, ptr, src, coef, bits)
         ref = oracle.reassemble_quant(x, g, None, 1e-5, ptr, src, coef, bits, want_pre=True)
         parity.check_activation_codes(got["codes"], got["scale"], got["zero"], got["rowsum"], ref, bits)
+
+
+def test_direct_call_keeps_its_compiled_map_only_while_the_contents_stay():
+    """The direct entry point keeps the compiled form of the last map it saw on a stream and recognises it by a
+    hash of the contents (map, gamma, beta), not by the pointers: calls on the same device arrays must follow the
+    arrays when they are rewritten in place, and calls with another channel count in between must not leave a
+    stale image behind."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    rng = np.random.default_rng(23)
+    M, bits = 29, 4
+
+    def case(C, shift):
+        # a map as the builder makes them: where c % 8 == shift, channels c and c + 1 are merged into row c
+        # (Eq. 4) and channel c + 2 is split into two sub-channels, rows c + 1 and c + 2 (Eq. 3, T = 2)
+        rows = []
+        for c in range(C):
+            k = (c - shift) % 8
+            rows.append([(c, 0.5), (c + 1, 0.5)] if k == 0 else [(c + 1, 0.5)] if k == 1 else [(c, 0.5)] if k == 2 else [(c, 1.0)])
+        ptr = np.zeros(C + 1, np.int32)
+        ptr[1:] = np.cumsum([len(r) for r in rows])
+        src = np.array([sj for r in rows for sj, _ in r], np.int32)
+        coef = np.array([cj for r in rows for _, cj in r], np.float32)
+        return ptr, src, coef
+
+    bufs = {}
+    for C in (4096, 5120):
+        x = synth.f32_to_bf16_bits((rng.standard_normal((M, C)) * (1 + 20 * (rng.random(C) < 0.01))).astype(np.float32))
+        g = (1 + 0.1 * rng.standard_normal(C)).astype(np.float32)
+        ptr, src, coef = case(C, 0)
+        bufs[C] = dict(x=x, xd=G.dev_x(x), g=g, gd=G.dev(g), ptr=ptr, src=src, coef=coef, pd=G.dev(ptr), sd=G.dev(src),
+                       cd=G.dev(coef), codes=torch.zeros((M, C // 2), dtype=torch.uint8, device=G.DEV),
+                       sc=torch.zeros(M, dtype=torch.float32, device=G.DEV), ze=torch.zeros(M, dtype=torch.float32, device=G.DEV),
+                       rs=torch.zeros(M, dtype=torch.int32, device=G.DEV))
+
+    def run_and_check(C):
+        b = bufs[C]
+        B.qllm_reassemble_quant(b["xd"], b["gd"], None, b["pd"], b["sd"], b["cd"], bits, b["codes"], b["sc"], b["ze"], b["rs"])
+        torch.cuda.synchronize()
+        ref = oracle.reassemble_quant(b["x"], b["g"], None, 1e-5, b["ptr"], b["src"], b["coef"], bits, want_pre=True)
+        parity.check_activation_codes(synth.unpack_nibbles(b["codes"].cpu().numpy()), b["sc"].cpu().numpy(), b["ze"].cpu().numpy(),
+                                      b["rs"].cpu().numpy(), ref, bits)
+
+    run_and_check(4096)
+    run_and_check(4096)                                   # same contents: the image in place serves
+    b = bufs[4096]
+    # same pointers, same sizes, other contents: another set of merged rows ...
+    b["ptr"], b["src"], b["coef"] = case(4096, 3)
+    assert b["src"].size == b["sd"].numel()
+    b["pd"].copy_(torch.from_numpy(b["ptr"])); b["sd"].copy_(torch.from_numpy(b["src"])); b["cd"].copy_(torch.from_numpy(b["coef"]))
+    run_and_check(4096)
+    # ... one coefficient ...
+    b["coef"] = b["coef"].copy(); b["coef"][5] *= 0.75
+    b["cd"].copy_(torch.from_numpy(b["coef"]))
+    run_and_check(4096)
+    # ... and one gamma
+    b["g"] = b["g"].copy(); b["g"][77] = -1.5
+    b["gd"].copy_(torch.from_numpy(b["g"]))
+    run_and_check(4096)
+    # another channel count on the same stream in between, then the first again
+    run_and_check(5120)
+    run_and_check(4096)
+    run_and_check(5120)
