@@ -53,26 +53,44 @@ __device__ __forceinline__ void eq2_params(float lo, float hi, float qmax, float
     zero = -rintf(lo * inv);
 }
 
+// How a row's codes are made from its Eq. 2 parameters.  round(f / alpha) + zero is taken as the low bits of
+// fma(f, 1 / alpha, 1.5 * 2^23) plus an integer constant (one rounding, to nearest even, no conversion
+// instruction: those run at a sixteenth of the arithmetic rate and would bound the kernel); quotients or
+// zero-points too large for that constant take the plain form.
+struct RowQuant {
+    float inv, zero, qmax;
+    int zadd, top;
+    bool big;
+    __device__ __forceinline__ RowQuant(float lo, float hi, float inv_, float zero_, float qmax_)
+        : inv(inv_), zero(zero_), qmax(qmax_), zadd(int(zero_) - kMagicBits), top(int(qmax_)),
+          big(fmaxf(fabsf(lo), fabsf(hi)) * inv_ >= 2097152.f || fabsf(zero_) >= 2097152.f) {}
+};
+
 // 8 codes of consecutive channels -> stored (4 bit: one 32-bit word, else two); returns their sum
-__device__ __forceinline__ int store_codes8(const float (&f)[8], float inv, float zero, float qmax, int bits,
-                                            uint8_t* out_row, int g) {
-    int n[8], sum = 0;
+__device__ __forceinline__ int store_codes8(const float (&f)[8], const RowQuant& q, int bits, uint8_t* out_row, int g) {
+    int n[8];
+    if (!q.big) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        n[j] = int(fminf(fmaxf(rintf(f[j] * inv) + zero, 0.f), qmax));
-        sum += n[j];
+        for (int j = 0; j < 8; ++j) n[j] = __float_as_int(fmaf(f[j], q.inv, kMagic)) + q.zadd;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) n[j] = int(fminf(fmaxf(rintf(f[j] * q.inv) + q.zero, 0.f), q.qmax));
     }
     if (bits == 4) {
-        uint32_t p = 0;
+        uint32_t p = 0;                                    // saturating packs clamp to 0 .. 15
 #pragma unroll
-        for (int j = 0; j < 8; ++j) p |= uint32_t(n[j]) << (4 * j);
+        for (int k = 3; k >= 0; --k) p = pack_sat_u4(n[2 * k + 1], n[2 * k], p);
         reinterpret_cast<uint32_t*>(out_row)[g] = p;
-    } else {
-        reinterpret_cast<uint2*>(out_row)[g] =
-            make_uint2(uint32_t(n[0]) | uint32_t(n[1]) << 8 | uint32_t(n[2]) << 16 | uint32_t(n[3]) << 24,
-                       uint32_t(n[4]) | uint32_t(n[5]) << 8 | uint32_t(n[6]) << 16 | uint32_t(n[7]) << 24);
+        const uint32_t nib = (p & 0x0F0F0F0Fu) + ((p >> 4) & 0x0F0F0F0Fu);
+        return int(__dp4a(nib, 0x01010101u, 0u));
     }
-    return sum;
+    // saturating packs clamp to 0 .. 255; 6-bit codes are cut at 63 first
+    uint32_t p0 = pack_sat_u8(min(n[3], q.top), min(n[2], q.top), 0u);
+    p0 = pack_sat_u8(min(n[1], q.top), min(n[0], q.top), p0);
+    uint32_t p1 = pack_sat_u8(min(n[7], q.top), min(n[6], q.top), 0u);
+    p1 = pack_sat_u8(min(n[5], q.top), min(n[4], q.top), p1);
+    reinterpret_cast<uint2*>(out_row)[g] = make_uint2(p0, p1);
+    return int(__dp4a(p1, 0x01010101u, __dp4a(p0, 0x01010101u, 0u)));
 }
 
 // WPR warps per row (1, 2, 4 or 8 of the CTA's 8), the row in registers: NVL vectors of 8 channels per lane.
@@ -120,6 +138,7 @@ quantize_rows_warp(const XT* __restrict__ x, int64_t M, int bits, uint8_t* __res
     const float qmax = float((1 << bits) - 1);
     float alpha, inv, zero;
     eq2_params(lo, hi, qmax, alpha, inv, zero);
+    const RowQuant rq(lo, hi, inv, zero, qmax);
     int sum = 0;
     if (live) {
         uint8_t* out_row = codes + m * (bits == 4 ? C / 2 : C);
@@ -127,7 +146,7 @@ quantize_rows_warp(const XT* __restrict__ x, int64_t M, int bits, uint8_t* __res
         for (int i = 0; i < NVL; ++i) {
             float f[8];
             v[i].get(f);
-            sum += store_codes8(f, inv, zero, qmax, bits, out_row, lane + 32 * (wsub + WPR * i));
+            sum += store_codes8(f, rq, bits, out_row, lane + 32 * (wsub + WPR * i));
         }
     }
     sum = __reduce_add_sync(0xffffffffu, sum);
