@@ -23,6 +23,29 @@ struct RowVec;                                             // 8 consecutive chan
 template <>
 struct RowVec<__nv_bfloat16> {
     uint4 r;
+    // running range of a lane's channels: bf16 pairs, compared as they are (no widening; a NaN operand is ignored)
+    struct Range {
+        __nv_bfloat162 lo, hi;
+        __device__ __forceinline__ Range() {
+            const uint32_t pinf = 0x7F807F80u, ninf = 0xFF80FF80u;
+            lo = *reinterpret_cast<const __nv_bfloat162*>(&pinf);
+            hi = *reinterpret_cast<const __nv_bfloat162*>(&ninf);
+        }
+        __device__ __forceinline__ void get(float& l, float& h) const {
+            const uint32_t a = *reinterpret_cast<const uint32_t*>(&lo), b = *reinterpret_cast<const uint32_t*>(&hi);
+            l = fminf(__uint_as_float(a << 16), __uint_as_float(a & 0xFFFF0000u));
+            h = fmaxf(__uint_as_float(b << 16), __uint_as_float(b & 0xFFFF0000u));
+        }
+    };
+    __device__ __forceinline__ void widen(Range& g) const {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const __nv_bfloat162 p = *reinterpret_cast<const __nv_bfloat162*>(&w[k]);
+            g.lo = __hmin2(g.lo, p);
+            g.hi = __hmax2(g.hi, p);
+        }
+    }
     __device__ __forceinline__ void load(const __nv_bfloat16* p) { r = __ldcs(reinterpret_cast<const uint4*>(p)); }
     __device__ __forceinline__ void get(float (&f)[8]) const {
         const uint32_t w[4] = {r.x, r.y, r.z, r.w};
@@ -36,6 +59,14 @@ struct RowVec<__nv_bfloat16> {
 template <>
 struct RowVec<float> {
     float4 a, b;
+    struct Range {
+        float lo = INFINITY, hi = -INFINITY;
+        __device__ __forceinline__ void get(float& l, float& h) const { l = lo; h = hi; }
+    };
+    __device__ __forceinline__ void widen(Range& g) const {
+        g.lo = min3(g.lo, a.x, a.y); g.lo = min3(g.lo, a.z, a.w); g.lo = min3(g.lo, b.x, b.y); g.lo = min3(g.lo, b.z, b.w);
+        g.hi = max3(g.hi, a.x, a.y); g.hi = max3(g.hi, a.z, a.w); g.hi = max3(g.hi, b.x, b.y); g.hi = max3(g.hi, b.z, b.w);
+    }
     __device__ __forceinline__ void load(const float* p) {
         a = __ldcs(reinterpret_cast<const float4*>(p));
         b = __ldcs(reinterpret_cast<const float4*>(p) + 1);
@@ -113,16 +144,10 @@ quantize_rows_warp(const XT* __restrict__ x, int64_t M, int bits, uint8_t* __res
     if (live) {
 #pragma unroll
         for (int i = 0; i < NVL; ++i) v[i].load(xr + 8 * (lane + 32 * (wsub + WPR * i)));
+        typename RowVec<XT>::Range range;
 #pragma unroll
-        for (int i = 0; i < NVL; ++i) {
-            float f[8];
-            v[i].get(f);
-#pragma unroll
-            for (int j = 0; j < 8; j += 2) {
-                lo = min3(lo, f[j], f[j + 1]);
-                hi = max3(hi, f[j], f[j + 1]);
-            }
-        }
+        for (int i = 0; i < NVL; ++i) v[i].widen(range);
+        range.get(lo, hi);
     }
     lo = redux_min(lo);
     hi = redux_max(hi);
