@@ -455,7 +455,8 @@ def run_fold(args):
         "gpu_launches": int(launches), "clocks": clocks,
         "roofline": {"kernel": "quantize_rows_warp", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS,
-                     "peak_source": f"{peaks['source']} STREAM-style copy", "bytes": nbytes, "traffic": None}}))
+                     "peak_source": f"{peaks['source']} STREAM-style copy", "bytes": nbytes,
+                     "traffic": _traffic("quantize_rows_warp", "c2_fold", M)}}))
 
 
 def launch_ranks(n, argv):
