@@ -75,3 +75,35 @@ def test_quantize_rows_alone(M, C, dtype, bits):
         parity.check_activation_codes(got, sc.cpu().numpy(), ze.cpu().numpy(), rs.cpu().numpy(), ref, bits)
     finally:
         parity.FLIP_BAND = old
+
+
+def test_quantize_rows_far_from_zero():
+    """A row far from zero with a tiny range (quotients of ~1.5e7, zero-point of the same size): fp32 cannot resolve
+    the oracle's decisions there, so the check is on what must hold whatever the rounding: codes inside the range, the
+    row sum of exactly those codes, alpha from the row's range, and every value reproduced to within a few steps."""
+    import torch
+    import gpu_util as G
+    from paper_2310_08041_b200 import binding as B
+    C, bits = 4096, 4
+    rng = np.random.default_rng(11)
+    x = np.zeros((4, C), np.float32)
+    x[0] = 1000.0 + 1e-3 * rng.random(C)
+    x[1] = -2500.0 + 4e-3 * rng.random(C)
+    x[2] = rng.standard_normal(C)                        # an ordinary row beside them
+    x[3] = 1000.0
+    codes = torch.zeros((4, C // 2), dtype=torch.uint8, device=G.DEV)
+    sc = torch.zeros(4, device=G.DEV); ze = torch.zeros(4, device=G.DEV); rs = torch.zeros(4, dtype=torch.int32, device=G.DEV)
+    B.qllm_quantize_rows(G.dev(x), bits, codes, sc, ze, rs)
+    torch.cuda.synchronize()
+    q = parity.unpack_codes(codes.cpu().numpy(), 4).astype(np.int64)
+    alpha, zero = sc.cpu().numpy().astype(np.float64), ze.cpu().numpy().astype(np.float64)
+    assert q.min() >= 0 and q.max() <= 15
+    assert np.array_equal(q.sum(1), rs.cpu().numpy())
+    x64 = x.astype(np.float64)
+    for m in range(3):
+        np.testing.assert_allclose(alpha[m], (x64[m].max() - x64[m].min()) / 15, rtol=2e-5)
+        assert zero[m] == np.rint(zero[m])
+        assert np.abs(x64[m] - alpha[m] * (q[m] - zero[m])).max() <= 2.5 * alpha[m] + 2e-4 * abs(x64[m]).max() * (m < 2)
+    assert alpha[3] == 1000.0 and np.all(q[3] == 0)
+    ref = oracle.quant_rows(x64[2:3], bits, want_pre=True)
+    parity.check_activation_codes(q[2:3].astype(np.uint8), sc.cpu().numpy()[2:3], ze.cpu().numpy()[2:3], rs.cpu().numpy()[2:3], ref, bits)
