@@ -82,22 +82,53 @@ rowsum_kernel(const uint8_t* __restrict__ codes, int64_t M, int K, int bits, int
     if (lane == 0) rowsum[m] = s;
 }
 
-// Packed nibbles [rows][K/2] -> byte codes [rows][K] in natural K order.  One 16-byte chunk
-// (32 codes) per thread in, 32 contiguous bytes out; purely bandwidth-bound.
+// Packed nibbles [rows][K/2] -> byte codes [rows][K] in natural K order.  A 16-byte chunk (32 codes) becomes 32
+// contiguous bytes; purely bandwidth-bound.  The kernel often runs beside a kernel that leaves it few warps per
+// SM, so a thread keeps kExpandUnroll loads in flight, and a lane pair swaps halves so that every store instruction
+// of a warp writes whole 32-byte sectors instead of half of each.
+constexpr int kExpandUnroll = 4;
+__device__ __forceinline__ void expand_chunk(const uint4& w, uint32_t (&o)[8]) {
+    const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t lo = in[k] & 0x0F0F0F0Fu, hi = (in[k] >> 4) & 0x0F0F0F0Fu;
+        o[2 * k] = __byte_perm(lo, hi, 0x5140);
+        o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);
+    }
+}
 __global__ void __launch_bounds__(256)
 expand_codes_kernel(const uint4* __restrict__ packed, int64_t chunks, uint4* __restrict__ bytes) {
-    for (int64_t i = int64_t(blockIdx.x) * 256 + threadIdx.x; i < chunks; i += int64_t(gridDim.x) * 256) {
-        const uint4 w = packed[i];
-        const uint32_t in[4] = {w.x, w.y, w.z, w.w};
-        uint32_t o[8];
+    const int lane = threadIdx.x & 31;
+    const bool odd = lane & 1;
+    const int64_t step = int64_t(gridDim.x) * 256;
+    // whole warps stay in the loop (the exchange below needs both lanes of a pair); chunks beyond the end are
+    // loaded as zeros and not stored
+    const int64_t first = int64_t(blockIdx.x) * 256 + (threadIdx.x & ~31);
+    for (int64_t i0 = first; i0 < chunks; i0 += step * kExpandUnroll) {
+        uint4 w[kExpandUnroll];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const uint32_t lo = in[k] & 0x0F0F0F0Fu, hi = (in[k] >> 4) & 0x0F0F0F0Fu;
-            o[2 * k] = __byte_perm(lo, hi, 0x5140);
-            o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);
+        for (int u = 0; u < kExpandUnroll; ++u) {
+            const int64_t i = i0 + u * step + lane;
+            w[u] = i < chunks ? __ldcs(packed + i) : make_uint4(0u, 0u, 0u, 0u);
         }
-        bytes[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
-        bytes[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+#pragma unroll
+        for (int u = 0; u < kExpandUnroll; ++u) {
+            const int64_t i = i0 + u * step + lane;
+            uint32_t o[8];
+            expand_chunk(w[u], o);
+            // even lane: keeps its first half, takes the odd lane's first half; odd lane: takes the even lane's
+            // second half, keeps its own second half.  Store 1 then covers the even lane's chunk, store 2 the odd's.
+            uint32_t a[4], b[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t got = __shfl_xor_sync(0xffffffffu, odd ? o[k] : o[4 + k], 1);
+                a[k] = odd ? got : o[k];                     // 16 bytes of the even lane's chunk
+                b[k] = odd ? o[4 + k] : got;                 // 16 bytes of the odd lane's chunk
+            }
+            const int64_t ie = i & ~int64_t(1);              // the pair's even chunk
+            if (ie < chunks) bytes[2 * ie + (odd ? 1 : 0)] = make_uint4(a[0], a[1], a[2], a[3]);
+            if (ie + 1 < chunks) bytes[2 * ie + 2 + (odd ? 1 : 0)] = make_uint4(b[0], b[1], b[2], b[3]);
+        }
     }
 }
 
@@ -106,7 +137,8 @@ expand_codes_kernel(const uint4* __restrict__ packed, int64_t chunks, uint4* __r
 int launch_expand_codes(const uint8_t* packed, int64_t rows, int K, uint8_t* bytes, cudaStream_t st) {
     const int64_t chunks = rows * (K / 32);
     if (chunks == 0) return QLLM_OK;
-    const int grid = int(std::min<int64_t>((chunks + 255) / 256, int64_t(device_sm_count()) * 16));
+    const int64_t per_cta = 256 * kExpandUnroll;
+    const int grid = int(std::min<int64_t>((chunks + per_cta - 1) / per_cta, int64_t(device_sm_count()) * 16));
     expand_codes_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const uint4*>(packed), chunks,
                                               reinterpret_cast<uint4*>(bytes));
     return after_launch();
