@@ -122,6 +122,10 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t full_addr0 = ptx::map_to_cta(ptx::smem_addr(&full[0]), 0);
             uint32_t it = 0;
             bool ok = true;
+            // The kernel is launched as a programmatic dependent of the kernel before it on the stream (for a layer,
+            // the pre-GEMM kernel that writes the tokens): all of the set-up above has run under that kernel's tail
+            // and the launch latency; the roles that touch global memory wait here for it to be complete.
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int tile = pair; ok && tile < num_tiles; tile += npairs) {
                 const int m0 = (tile % tiles_m) * 2 * BM + int(rank) * BM;
                 const int n0 = (tile / tiles_m) * BN + int(rank) * T::HALF_N;
@@ -197,6 +201,7 @@ qgemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                            ptx::map_to_cta(ptx::smem_addr(&acc_empty[1]), 0)};
         uint8_t* mybuf = outbuf + (warp - kFirstEpiWarp) * 2048;
         uint32_t lt = 0;
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // the row terms below come from the kernel before
         for (int tile = pair; tile < num_tiles; tile += npairs, ++lt) {
             const uint32_t abuf = lt & 1, aph = (lt >> 1) & 1;
             const int m0 = (tile % tiles_m) * 2 * BM + int(rank) * BM;
@@ -276,13 +281,15 @@ int launch_pair(const uint8_t* a, const uint8_t* w, int64_t M, int N, int K, con
     cfg.blockDim = dim3(T::THREADS);
     cfg.dynamicSmemBytes = T::SMEM;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     QLLM_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmW, tmO, M, N, K, ep, status));
     return after_launch();
 }
