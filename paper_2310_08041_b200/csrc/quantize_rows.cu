@@ -37,7 +37,7 @@ struct RowVec<__nv_bfloat16> {
             h = fmaxf(__uint_as_float(b << 16), __uint_as_float(b & 0xFFFF0000u));
         }
     };
-    __device__ __forceinline__ void widen(Range& g) const {
+    __device__ __forceinline__ void extend(Range& g) const {
         const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -63,7 +63,7 @@ struct RowVec<float> {
         float lo = INFINITY, hi = -INFINITY;
         __device__ __forceinline__ void get(float& l, float& h) const { l = lo; h = hi; }
     };
-    __device__ __forceinline__ void widen(Range& g) const {
+    __device__ __forceinline__ void extend(Range& g) const {
         g.lo = min3(g.lo, a.x, a.y); g.lo = min3(g.lo, a.z, a.w); g.lo = min3(g.lo, b.x, b.y); g.lo = min3(g.lo, b.z, b.w);
         g.hi = max3(g.hi, a.x, a.y); g.hi = max3(g.hi, a.z, a.w); g.hi = max3(g.hi, b.x, b.y); g.hi = max3(g.hi, b.z, b.w);
     }
@@ -146,7 +146,7 @@ quantize_rows_warp(const XT* __restrict__ x, int64_t M, int bits, uint8_t* __res
         for (int i = 0; i < NVL; ++i) v[i].load(xr + 8 * (lane + 32 * (wsub + WPR * i)));
         typename RowVec<XT>::Range range;
 #pragma unroll
-        for (int i = 0; i < NVL; ++i) v[i].widen(range);
+        for (int i = 0; i < NVL; ++i) v[i].extend(range);
         range.get(lo, hi);
     }
     lo = redux_min(lo);
