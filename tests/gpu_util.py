@@ -23,17 +23,41 @@ def bf16_bits(t):
     return t.view(torch.int16).cpu().numpy().view(np.uint16)
 
 
+class Guarded:
+    """An output tensor placed in the middle of a larger buffer filled with a canary pattern: check() fails when a
+    kernel wrote a byte before or behind the tensor it was given."""
+    PAD = 4096                                           # bytes on either side (keeps the 16-byte alignment)
+
+    def __init__(self, shape, dtype, fill):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.raw = torch.full((n + 2 * self.PAD,), 0x5C, dtype=torch.uint8, device=DEV)
+        self.n = n
+        self.t = self.raw[self.PAD:self.PAD + n].view(dtype).view(*shape)
+        self.t.fill_(fill)
+
+    def check(self, what="output"):
+        r = self.raw.cpu().numpy()
+        before, after = r[:self.PAD], r[self.PAD + self.n:]
+        assert (before == 0x5C).all(), f"{what}: {int((before != 0x5C).sum())} bytes written in front of the tensor"
+        assert (after == 0x5C).all(), f"{what}: {int((after != 0x5C).sum())} bytes written behind the tensor"
+
+
 def run_reassemble_quant(x_np, gamma, beta, eps, ptr, src, coef, bits, want_rowsum=True):
     x = dev_x(x_np)
     M, C = x.shape
     row = C // 2 if bits == 4 else C
-    codes = torch.full((M, row), 0xAB, dtype=torch.uint8, device=DEV)
-    a_scale = torch.full((M,), -1.0, dtype=torch.float32, device=DEV)
-    a_zero = torch.full((M,), -1e9, dtype=torch.float32, device=DEV)
-    a_rowsum = torch.full((M,), -7, dtype=torch.int32, device=DEV) if want_rowsum else None
+    g_codes = Guarded((M, row), torch.uint8, 0xAB)
+    g_scale = Guarded((M,), torch.float32, -1.0)
+    g_zero = Guarded((M,), torch.float32, -1e9)
+    g_rowsum = Guarded((M,), torch.int32, -7) if want_rowsum else None
+    codes, a_scale, a_zero = g_codes.t, g_scale.t, g_zero.t
+    a_rowsum = g_rowsum.t if want_rowsum else None
     B.qllm_reassemble_quant(x, None if gamma is None else dev(gamma), None if beta is None else dev(beta), dev(ptr), dev(src), dev(coef),
                             bits, codes, a_scale, a_zero, a_rowsum, ln_eps=eps)
     torch.cuda.synchronize()
+    g_codes.check("codes"); g_scale.check("a_scale"); g_zero.check("a_zero")
+    if g_rowsum is not None:
+        g_rowsum.check("a_rowsum")
     stored = codes.cpu().numpy()
     return dict(stored=stored, codes=synth.unpack_nibbles(stored) if bits == 4 else stored,
                 scale=a_scale.cpu().numpy(), zero=a_zero.cpu().numpy(),

@@ -62,10 +62,13 @@ def test_quantize_rows_alone(M, C, dtype, bits):
     else:
         x64 = x.astype(np.float64)
         xd = G.dev(x)
-    codes = torch.full((M, C // 2 if bits == 4 else C), 0xAB, dtype=torch.uint8, device=G.DEV)
-    sc = torch.zeros(M, device=G.DEV); ze = torch.zeros(M, device=G.DEV); rs = torch.zeros(M, dtype=torch.int32, device=G.DEV)
+    guards = [G.Guarded((M, C // 2 if bits == 4 else C), torch.uint8, 0xAB), G.Guarded((M,), torch.float32, 0),
+              G.Guarded((M,), torch.float32, 0), G.Guarded((M,), torch.int32, 0)]
+    codes, sc, ze, rs = (g.t for g in guards)
     B.qllm_quantize_rows(xd, bits, codes, sc, ze, rs)
     torch.cuda.synchronize()
+    for g, what in zip(guards, ("codes", "a_scale", "a_zero", "a_rowsum")):
+        g.check(what)
     got = codes.cpu().numpy()
     got = parity.unpack_codes(got, 4) if bits == 4 else got
     ref = oracle.quant_rows(x64, bits, want_pre=True)

@@ -39,10 +39,12 @@ def test_accumulators_bit_exact(M, N, K, a_bits, w_bits):
     from paper_2310_08041_b200 import binding as B
     qa, qw = _operands(M + N + K, M, N, K, a_bits, w_bits)
     ref = oracle.int_matmul(qa, qw)
-    acc = torch.full((M, N), -12345, dtype=torch.int32, device=G.DEV)
+    guard = G.Guarded((M, N), torch.int32, -12345)       # canaries on both sides of the output
+    acc = guard.t
     B.qllm_qgemm_acc(G.dev(G.store_codes(qa, a_bits)), G.dev(G.store_codes(qw, w_bits)), acc, M, N, K, a_bits, w_bits)
     torch.cuda.synchronize()
     assert B.qllm_poll_status() == 0
+    guard.check("accumulators")
     assert np.array_equal(acc.cpu().numpy(), ref)
 
 
@@ -74,12 +76,14 @@ def test_epilogue_matches_oracle(M, N, K, a_bits, w_bits, out_dtype):
     for bias in (e["bias"], None):
         for give_rowsum in (True, False):
             ref = oracle.epilogue(acc, K, e["a_scale"], e["a_zero"], e["a_rowsum"], e["w_scale"], e["w_zero"], e["w_colsum"], bias)
-            out = torch.zeros((M, N), dtype=tdt, device=G.DEV)
+            guard = G.Guarded((M, N), tdt, 0)
+            out = guard.t
             B.qllm_qgemm(da, G.dev(e["a_scale"]), G.dev(e["a_zero"]), dw, G.dev(e["w_scale"]), G.dev(e["w_zero"]),
                          G.dev(e["w_colsum"]), None if bias is None else G.dev(bias), out, M, N, K, a_bits, w_bits,
                          a_rowsum=G.dev(e["a_rowsum"]) if give_rowsum else None)
             torch.cuda.synchronize()
-            got = out.cpu().numpy() if out_dtype == "f32" else G.bf16_bits(out)
+            guard.check("out")
+            got = out.cpu().numpy() if out_dtype == "f32" else G.bf16_bits(out.contiguous())
             parity.check_output(got, ref, out_dtype)
 
 
