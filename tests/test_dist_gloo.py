@@ -82,3 +82,27 @@ def test_bench_gpus_flag_starts_that_many_ranks():
     r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "4", "--steps", "1", "--warmup", "1", "--stub"],
                        capture_output=True, text=True, timeout=120, env=env2)
     assert r.returncode != 0 and not [l for l in r.stdout.splitlines() if l.startswith("{")]
+
+
+def test_traffic_record_is_tied_to_the_kernel_sources(tmp_path, monkeypatch):
+    """bench.py takes roofline.traffic from a `traffic-record:` line of a profile summary only while the kernel's
+    sources still hash to what the line recorded; a changed source, another workload or another M give None."""
+    import hashlib
+    import bench
+    src_dir = tmp_path / "paper_2310_08041_b200" / "csrc"
+    src_dir.mkdir(parents=True)
+    (tmp_path / "profiles").mkdir()
+    (src_dir / "k.cu").write_text("kernel v1\n")
+    (src_dir / "h.cuh").write_text("header\n")
+    sha = hashlib.sha256(b"kernel v1\n" + b"header\n").hexdigest()[:16]
+    (tmp_path / "profiles" / "k.md").write_text(
+        "# some kernel\n\ntraffic-record: kernel=k_kernel workload=w1 M=64 bytes=123456 sources=k.cu,h.cuh sha256=%s\n" % sha)
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    assert bench._traffic("k_kernel", "w1", 64) == 123456.0
+    assert bench._traffic("k_kernel", "w1", 65) is None
+    assert bench._traffic("k_kernel", "w2", 64) is None
+    assert bench._traffic("other", "w1", 64) is None
+    (src_dir / "k.cu").write_text("kernel v2\n")
+    assert bench._traffic("k_kernel", "w1", 64) is None
+    (src_dir / "k.cu").unlink()
+    assert bench._traffic("k_kernel", "w1", 64) is None
